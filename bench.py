@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the suffix-automaton draft + greedy-verify step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+
+One "step" = one closed-loop iteration of the whole hot path over one batch: vocabulary argmax
+over [B, K+1, V] bf16 logits, prefix accept, automaton walk over the accepted tokens, next draft
+(`sam_step`).  The workload is synthetic (see workload/agent_memory.py); the default is the
+B=256, K=16, 16M-token-corpus configuration.  Prints ONE JSON line on rank 0.
+
+Timing: every step is bracketed by CUDA events on the launching stream; the stand-in target
+model (sparse planting of the wanted tokens into the resident noise logits between steps) is
+outside the events.  `--impl reference` times the CPU oracle instead (host cores, wall clock).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workload as W  # noqa: E402
+
+METRIC = "sam_draft_verify_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the current kernel)
+NCU_DRAM_BYTES_PER_ROW = None
+
+
+# ----------------------------------------------------------------------------- helpers
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_over_ranks(tokens: int, ms: float, world: int, backend_device=None):
+    """(sum of tokens, max of milliseconds) over all ranks; identity when world == 1."""
+    if world == 1:
+        return tokens, ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(tokens)], dtype=torch.float64, device=backend_device)
+    m = torch.tensor([float(ms)], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    dist.all_reduce(m, op=dist.ReduceOp.MAX)
+    return int(round(t.item())), float(m.item())
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.lines = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_inputs_gpu(cfg, device):
+    """Corpus (host) and the noise logits generated on the device (seeded torch generator)."""
+    import torch
+    corpus = W.make_corpus(cfg)
+    g = torch.Generator(device=device)
+    g.manual_seed(1000 + cfg.seed)
+    R = cfg.rows
+    logits = torch.empty((R, cfg.vocab), dtype=torch.bfloat16, device=device)
+    blk = max(1, (1 << 26) // cfg.vocab)
+    for r0 in range(0, R, blk):
+        r1 = min(R, r0 + blk)
+        logits[r0:r1] = torch.randn((r1 - r0, cfg.vocab), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    rowmax = logits.max(dim=1).values.view(torch.int16).cpu().numpy().view(np.uint16)
+    return corpus, logits, rowmax
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2512_18337_b200 as S
+    from paper_2512_18337_b200.build import build
+    from tests.cuda_backend import CudaBackend
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    device = f"cuda:{local_rank}"
+    torch.cuda.set_device(device)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+
+    base = W.CONFIGS[args.config]
+    # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
+    # read-only automaton is replicated; no data-path collective
+    cfg = base.scaled(steps=args.warmup + args.steps + args.e2e_steps + 1)
+    stream_cfg = cfg.scaled(seed=cfg.seed + 7919 * rank) if rank > 0 else cfg
+
+    t0 = time.time()
+    corpus, logits, rowmax = make_inputs_gpu(cfg, device)
+    scripts = W.make_scripts(stream_cfg, corpus)
+    t_inputs = time.time() - t0
+    t0 = time.time()
+    index = S.SamIndex(corpus, [cfg.separator], device=device, upload=False)
+    t_build = time.time() - t0
+    t0 = time.time()
+    index.blob = torch.empty(index.device_bytes, dtype=torch.uint8, device=device)
+    S.sam_upload(index.handle, index.blob)
+    t_upload = time.time() - t0
+
+    feeder = W.ClosedLoopFeeder(stream_cfg, scripts, rowmax)
+    be = CudaBackend(cfg, corpus, logits, index=index, device=device)
+    toks, n = feeder.prime_tokens()
+    drafts, n_draft = be.prime(toks, n)
+
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    tokens = 0
+    stats_trace = []
+
+    def one_step(t, timed_slot=None):
+        nonlocal drafts, n_draft, tokens
+        ow = feeder.overwrites(t, drafts, n_draft)
+        keep = np.arange(ow["row"].shape[0])
+        saved = be.poke(ow["row"], ow["col"], ow["bits"], keep)
+        in_nd = n_draft
+        if timed_slot is not None:
+            ev[timed_slot][0].record()
+            be.launch_step()
+            ev[timed_slot][1].record()
+        else:
+            be.launch_step()
+        torch.cuda.synchronize()
+        n_acc = be.n_accepted.cpu().numpy()
+        drafts, n_draft = be.drafts.cpu().numpy(), be.n_draft.cpu().numpy()
+        be.unpoke(ow["row"], ow["col"], saved)
+        feeder.advance(n_acc)
+        if timed_slot is not None:
+            tokens += int(n_acc.sum())
+            stats_trace.append(dict(n_accepted=n_acc, in_n_draft=in_nd))
+
+    for t in range(args.warmup):
+        one_step(t)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    S.sam_profile_enable(args.steps)
+    wall0 = time.time()
+    for i in range(args.steps):
+        one_step(args.warmup + i, timed_slot=i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    wall = time.time() - wall0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    prof = [S.sam_profile_read(i) for i in range(S.sam_profile_count())]
+    S.sam_profile_enable(0)
+    total_ms = float(sum(step_ms))
+    argmax_ms = statistics.mean(p[0] for p in prof)
+    accept_ms = statistics.mean(p[1] for p in prof)
+
+    # ---- end to end through the host-buffer entry point: logits and bookkeeping start in pinned host memory
+    e2e = None
+    if args.e2e_steps > 0:
+        B, K, V = cfg.B, cfg.K, cfg.vocab
+        host_logits = torch.empty(logits.shape, dtype=torch.bfloat16).pin_memory()
+        host_logits.copy_(logits)
+        torch.cuda.synchronize()
+        hraw = host_logits.view(torch.int16).numpy().view(np.uint16)
+        i32 = dict(dtype=torch.int32)
+        h = {k: torch.zeros(s, **i32).pin_memory() for k, s in dict(
+            drafts=(B, K), n_draft=(B,), argmax=(B, K + 1), accepted=(B, K + 1), n_accepted=(B,),
+            state=(B,), mlen=(B,)).items()}
+        h["drafts"].copy_(be.drafts)
+        h["n_draft"].copy_(be.n_draft)
+        h["state"].copy_(be.state)
+        h["mlen"].copy_(be.mlen)
+        torch.cuda.synchronize()
+        sb = S.sam_step_host_staging_bytes(V, B, K, V)
+        staging = torch.empty(sb, dtype=torch.uint8, device=device)
+        e2e_tokens, e2e_s = 0, 0.0
+        for i in range(args.e2e_steps):
+            t = args.warmup + args.steps + i
+            ow = feeder.overwrites(t, h["drafts"].numpy(), h["n_draft"].numpy())
+            saved = hraw[ow["row"], ow["col"]].copy()
+            hraw[ow["row"], ow["col"]] = ow["bits"]
+            torch.cuda.synchronize()
+            c0 = time.perf_counter()
+            S.sam_step_host(index.handle, host_logits, V, B, K, V, h["drafts"], h["n_draft"], h["argmax"],
+                            h["accepted"], h["n_accepted"], h["state"], h["mlen"], cfg.min_match,
+                            h["drafts"], h["n_draft"], staging, sb)
+            c1 = time.perf_counter()
+            hraw[ow["row"], ow["col"]] = saved
+            n_acc = h["n_accepted"].numpy().copy()
+            feeder.advance(n_acc)
+            if i > 0 or args.e2e_steps == 1:       # first host step warms the pinned path
+                e2e_tokens += int(n_acc.sum())
+                e2e_s += c1 - c0
+        h2d = logits.numel() * 2 + (B * K + 3 * B) * 4
+        d2h = (2 * B * (K + 1) + B * K + 4 * B) * 4
+        e2e_tokens, e2e_ms = reduce_over_ranks(e2e_tokens, e2e_s * 1e3, world, device)
+        e2e = {"value": e2e_tokens / (e2e_ms / 1e3) if e2e_ms > 0 else None, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": max(1, args.e2e_steps - 1), "api": "sam_step_host (pinned host buffers, wall clock incl. sync)"}
+        del staging, host_logits
+
+    all_tokens, max_ms = reduce_over_ranks(tokens, total_ms, world, device)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    R = cfg.rows
+    alg_bytes = R * (2 * cfg.vocab + 4)
+    achieved = alg_bytes / (argmax_ms * 1e-3) / 1e9
+    st = W.trace_stats(cfg, stats_trace)
+    out = {
+        "metric": METRIC, "value": all_tokens / (max_ms / 1e3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.vocab, "min_match": cfg.min_match,
+                   "corpus_tokens": cfg.n_corpus, "accept_p": cfg.accept_p,
+                   "logits_bytes_per_step": R * cfg.vocab * 2,
+                   "l2": "inputs larger than L2 (logits re-read from HBM every step)" if R * cfg.vocab * 2 > 252e6
+                   else "inputs smaller than 2x L2: bandwidth figures are not HBM figures",
+                   "timing": "CUDA events around each sam_step on the launching stream, summed over steps; "
+                             "sparse logits planting between steps excluded"},
+        "steps_per_s": args.steps / (max_ms / 1e3),
+        "stream_steps_per_s": world * cfg.B * args.steps / (max_ms / 1e3),
+        "gpu_launches": 2 * args.steps,
+        "kernels_ms": {"argmax": argmax_ms, "accept_walk_draft": accept_ms},
+        "roofline": {"kernel": "argmax", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
+                     "traffic": (NCU_DRAM_BYTES_PER_ROW * R) if NCU_DRAM_BYTES_PER_ROW else None,
+                     "algorithmic_bytes": alg_bytes},
+        "walk": {"draft_tokens_per_s": st["mean_n_draft"] * cfg.B * args.steps / (accept_ms * args.steps / 1e3),
+                 "committed_tokens_per_s_kernel_only": tokens / (accept_ms * args.steps / 1e3)},
+        "ote": st["ote"], "shr": st["shr"], "mean_n_draft": st["mean_n_draft"],
+        "e2e": e2e, "clocks": clocks,
+        "setup_s": {"inputs": t_inputs, "sam_build": t_build, "sam_upload": t_upload,
+                    "sam_build_tokens_per_s": cfg.n_corpus / t_build,
+                    "states": index.n_states, "edges": index.n_edges, "device_bytes": index.device_bytes},
+        "wall_s_timed_loop_incl_harness": wall,
+    }
+    if args.cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(cfg, corpus, scripts, logits, rowmax, args.cpu_steps)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- oracle arm
+def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads):
+    """Times the oracle's step (wall clock, planting excluded) on the same closed loop."""
+    import oracle
+    from tests.oracle_backend import OracleBackend
+    feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    t0 = time.time()
+    be = OracleBackend(cfg, corpus, host_bits, threads)
+    t_build = time.time() - t0
+    toks, n = feeder.prime_tokens()
+    drafts, n_draft = be.prime(toks, n)
+    tokens, secs = 0, 0.0
+    for t in range(warmup + steps):
+        ow = feeder.overwrites(t, drafts, n_draft)
+        keep = np.arange(ow["row"].shape[0])
+        saved = be.poke(ow["row"], ow["col"], ow["bits"], keep)
+        c0 = time.perf_counter()
+        out = be.step(drafts, n_draft)
+        c1 = time.perf_counter()
+        be.unpoke(ow["row"], ow["col"], saved)
+        feeder.advance(out["n_accepted"])
+        drafts, n_draft = out["drafts"], out["n_draft"]
+        if t >= warmup:
+            tokens += int(out["n_accepted"].sum())
+            secs += c1 - c0
+    return tokens, secs, t_build
+
+
+def cpu_baseline(cfg, corpus, scripts, logits_dev, rowmax, steps):
+    import oracle
+    host_bits = logits_dev.view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+    threads = oracle.host_threads()
+    tokens, secs, t_build = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, 1, steps, threads)
+    return {"value": tokens / secs, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"all {cfg.B} streams, first {steps} closed-loop steps after 1 warm-up step "
+                      f"({secs:.2f} s of oracle stepping; oracle automaton build {t_build:.1f} s not included)",
+            "ms_per_step": secs / steps * 1e3,
+            "argmax_GBps": cfg.rows * cfg.vocab * 2 * steps / secs / 1e9}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    base = W.CONFIGS[args.config]
+    steps = min(args.steps, 40)
+    warmup = min(args.warmup, 3)
+    cfg = base.scaled(steps=warmup + steps + 1)
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    host_bits = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(host_bits).max(axis=1))
+    threads = oracle.host_threads()
+    tokens, secs, t_build = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads)
+    v = tokens / secs
+    sample = (f"all {cfg.B} streams of {cfg.name}, {steps} closed-loop steps per run after {warmup} warm-up "
+              f"(requested {args.steps}/{args.warmup}; capped so the run stays within minutes)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": secs / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.vocab, "min_match": cfg.min_match,
+                   "corpus_tokens": cfg.n_corpus},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "oracle_build_s": t_build,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (default: B=256, K=16)")
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--cpu-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

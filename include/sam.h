@@ -1,0 +1,192 @@
+/*
+ * sam.h - C ABI of the B200 (sm_100a) suffix-automaton draft + greedy-verify library.
+ *
+ * The operations are those of the AgentSAM speculative decoding loop (Section 5.4.2
+ * "Algorithm design", Section 5.4.3 "System design", Algorithm 3):
+ *   build the automaton over the context memory once (setup),
+ *   per decoding step: follow automaton transitions over the newly verified tokens and
+ *   emit a continuation of bounded length (draft), let the target model score the proposal
+ *   (its logits are an INPUT here), take the row-wise greedy choice, commit the longest
+ *   matching prefix plus the model's own token at the first mismatch (verify), and feed the
+ *   committed tokens straight back into the automaton walk (step).
+ *
+ * General rules
+ *   - Every function returns an int status: SAM_OK (0) or a negative SAM_ERR_* code.
+ *     Nothing throws, aborts or traps; device code never faults on out-of-vocabulary tokens.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA device memory of
+ *     the current device, allocated and owned by the caller (e.g. torch tensors).
+ *   - Hot-path calls (sam_draft, sam_verify, sam_step) only enqueue kernels on the given
+ *     stream (a cudaStream_t passed as void*, NULL = default stream).  They never allocate,
+ *     never synchronise and never copy to the host; outputs are valid once the stream reaches
+ *     the end of the enqueued work.
+ *   - Token ids are int32.  The per-stream state is the pair (state, matched_len), owned by
+ *     the caller; a new stream starts at (0, 0).
+ *   - There is no CPU fallback: without a usable CUDA device the hot-path calls fail with
+ *     SAM_ERR_CUDA.
+ */
+#ifndef SAM_B200_H
+#define SAM_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SAM_OK                 0
+#define SAM_ERR_INVALID_ARG   (-1)  /* null pointer, size out of range, misaligned pointer */
+#define SAM_ERR_NOMEM         (-2)  /* host allocation failed during sam_build */
+#define SAM_ERR_NOT_UPLOADED  (-3)  /* hot-path call before a successful sam_upload */
+#define SAM_ERR_CUDA          (-4)  /* a CUDA runtime call or kernel launch failed; see sam_last_cuda_error */
+#define SAM_ERR_TOO_SMALL     (-5)  /* caller buffer (device blob, workspace) smaller than required */
+
+#define SAM_K_MAX             32    /* largest draft length K accepted by the hot path */
+#define SAM_MAX_SEPARATORS    16    /* largest number of separator ids */
+
+typedef struct sam_index sam_index; /* opaque; owns the host-side automaton; device memory belongs to the caller */
+
+/* ---------------------------------------------------------------- setup (host, blocking) */
+
+/* Builds the suffix automaton of corpus[0..n) by the online, token-by-token construction
+ * (Section 5.4.3: incremental, linear in the context length).  States are numbered in
+ * creation order: root 0, then for each position the new state followed by its clone when a
+ * split happens; a clone copies transitions, suffix link and first end position.
+ * Separators are ordinary symbols for construction and for the walk; they only stop draft
+ * emission and are never emitted.
+ *   corpus      host, n int32 tokens, 1 <= n <= 2^29
+ *   separators  host, n_sep ids (0 <= n_sep <= SAM_MAX_SEPARATORS); may be NULL when n_sep = 0
+ *   out         receives the handle; release it with sam_free
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOMEM. */
+int sam_build(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep,
+              sam_index** out);
+
+/* Sizes of the built automaton and the byte size of the device blob sam_upload needs.
+ * Any output pointer may be NULL. */
+int sam_sizes(const sam_index* idx, int64_t* n_states, int64_t* n_edges, int64_t* device_bytes);
+
+/* Copies the automaton as flat host arrays (for inspection and parity checks):
+ *   len, link, firstpos  [n_states] int32  (root: 0, -1, -1; firstpos = smallest end position)
+ *   row_ptr              [n_states + 1] int64, CSR offsets into the edge arrays
+ *   edge_tok, edge_dst   [n_edges] int32, each row strictly ascending by token id
+ * All six are host buffers owned by the caller; any may be NULL to skip it. */
+int sam_export(const sam_index* idx, int32_t* len, int32_t* link, int32_t* firstpos,
+               int64_t* row_ptr, int32_t* edge_tok, int32_t* edge_dst);
+
+/* Packs the automaton and the corpus into the device layout and copies it into device_buf
+ * (device, 256-byte aligned, at least device_bytes from sam_sizes) with cudaMemcpyAsync on the
+ * stream, then synchronises that stream once (setup, not the hot path).  The handle remembers
+ * device_buf; the caller keeps it alive and unmodified while hot-path calls use the handle.
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_SMALL, SAM_ERR_CUDA, SAM_ERR_NOMEM. */
+int sam_upload(sam_index* idx, void* device_buf, int64_t bytes, void* cuda_stream);
+
+/* Releases the host-side automaton.  Device memory is the caller's. NULL is allowed. */
+void sam_free(sam_index* idx);
+
+/* ---------------------------------------------------------------- verification scratch */
+
+/* Bytes of device scratch sam_verify / sam_step need for B streams and draft length K
+ * (one 64-bit partial result per logits row).  Returns a negative SAM_ERR_* on bad sizes. */
+int64_t sam_workspace_bytes(int32_t B, int32_t K);
+
+/* Zero-fills the scratch (device, 8-byte aligned) on the stream.  Required once before the
+ * first sam_verify / sam_step that uses it; every successful call leaves it zeroed again.
+ * Call it again after a hot-path call returned an error.  Calls that share one workspace
+ * must not overlap on the device. */
+int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------- hot path (device, async) */
+
+/* Draft (Section 5.4.2; Algorithm 3 "FollowTransitions" and "Emit speculative tokens").
+ * For every stream b: consume new_tokens[b, 0..n_new[b]) from (state[b], matched_len[b]):
+ * a transition on the token extends the match by one; on a miss the suffix link is followed
+ * and the match shortened to that state's length, and a miss at the root resets the match to 0.
+ * Then, if matched_len[b] >= min_match, emit the tokens that follow the FIRST occurrence of
+ * the matched suffix in the corpus: up to K tokens, stopping before a separator or the corpus
+ * end; otherwise emit nothing.
+ *   B            streams, >= 0 (0 is a no-op)
+ *   state, matched_len   device [B] int32, in/out
+ *   new_tokens   device [B, ld] int32 row-major; n_new device [B] int32 with 0 <= n_new[b] <= ld
+ *                (values above ld are clamped to ld, negative to 0); n_new[b] = 0 re-emits the draft
+ *   K            1..SAM_K_MAX;  min_match >= 1
+ *   drafts       device [B, K] int32, unused slots = -1;  n_draft device [B] int32
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_CUDA. */
+int sam_draft(const sam_index* idx, int32_t B, int32_t* state, int32_t* matched_len,
+              const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
+              int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft,
+              void* cuda_stream);
+
+/* Greedy verification (Algorithm 3 "Validate with main LLM; commit matched prefix; fallback").
+ * logits row (b, j), j = 0..K, holds the target model's scores after the committed tokens and
+ * drafts[b, 0..j).  For all B*(K+1) rows: argmax over V bf16 values, the lowest index winning
+ * ties (-0 equals +0; a NaN never beats a number; a row whose element 0 is NaN yields 0).
+ * Then a = number of leading j < n_draft[b] with drafts[b,j] == argmax[b,j];
+ * accepted[b] = drafts[b,0..a) followed by argmax[b,a]; n_accepted[b] = a + 1.
+ *   logits_bf16       device, bf16, element (row r, column v) at logits_bf16[r*row_stride_elems + v],
+ *                     r = b*(K+1)+j; 2-byte aligned; read-only; fastest when rows are 16-byte aligned
+ *   row_stride_elems  >= V
+ *   drafts, n_draft   device [B,K], [B] (n_draft clamped to 0..K)
+ *   argmax_out        device [B, K+1] int32 (all rows, also those beyond n_draft)
+ *   accepted          device [B, K+1] int32, unused slots = -1;  n_accepted device [B] int32
+ *   workspace         device scratch of sam_workspace_bytes(B, K), zeroed by sam_workspace_init
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_SMALL, SAM_ERR_CUDA. */
+int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+               const int32_t* drafts, const int32_t* n_draft,
+               int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+               void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* Fused steady-state step (Algorithm 3, one iteration of the speculative decoding loop):
+ * sam_verify, then the accepted tokens of each stream are walked from (state, matched_len)
+ * exactly as sam_draft would with new_tokens = accepted, n_new = n_accepted, and the next
+ * draft is emitted - all on the device, with no host round trip in between.
+ * next_drafts / next_n_draft may alias drafts / n_draft.
+ * Errors: as sam_verify and sam_draft. */
+int sam_step(const sam_index* idx,
+             const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+             const int32_t* drafts, const int32_t* n_draft,
+             int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+             int32_t* state, int32_t* matched_len, int32_t min_match,
+             int32_t* next_drafts, int32_t* next_n_draft,
+             void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* Host-buffer form of sam_step, for callers whose logits and bookkeeping live in host memory
+ * (Algorithm 3, one loop iteration, end to end).  Copies logits [B*(K+1) rows, row_stride_elems
+ * apart, V used], drafts, n_draft, state and matched_len from the host into `staging`, runs
+ * sam_step there, copies argmax_out, accepted, n_accepted, state, matched_len, next_drafts and
+ * next_n_draft back and synchronises the stream before returning.  Every pointer except
+ * `staging` is HOST memory (pinned memory makes the copies asynchronous and faster); `staging`
+ * is device memory of at least sam_step_host_staging_bytes(...), 256-byte aligned, contents
+ * undefined between calls (it embeds the verification scratch, which the call zeroes itself).
+ * Errors: as sam_step. */
+int64_t sam_step_host_staging_bytes(int64_t row_stride_elems, int32_t B, int32_t K, int32_t V);
+int sam_step_host(const sam_index* idx,
+                  const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                  const int32_t* drafts, const int32_t* n_draft,
+                  int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                  int32_t* state, int32_t* matched_len, int32_t min_match,
+                  int32_t* next_drafts, int32_t* next_n_draft,
+                  void* staging, int64_t staging_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------- diagnostics */
+
+/* Per-kernel device timing of sam_verify / sam_step (measurement aid; the paper has no
+ * counterpart).  sam_profile_enable(n) creates CUDA events for the next n calls (n = 0 turns
+ * profiling off and frees them); while enabled, each call records events before the argmax
+ * kernel, between the two kernels and after the accept kernel on the caller's stream.
+ * sam_profile_read(i, ...) returns the two durations of the i-th profiled call in
+ * milliseconds; the stream must have been synchronised by the caller first.
+ * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
+int sam_profile_enable(int32_t max_calls);
+int32_t sam_profile_count(void);
+int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms);
+
+/* Static description of a status code. */
+const char* sam_strerror(int status);
+
+/* cudaError_t value of the most recent failed CUDA call made by this library on the calling
+ * thread (0 if none). */
+int sam_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAM_B200_H */

@@ -1,0 +1,261 @@
+"""ctypes binding of ``libsam_b200.so``: argument marshalling only.
+
+Function names and argument order follow ``include/sam.h``.  Device arguments are torch
+tensors (or raw integer addresses); host arguments are numpy arrays.  Every step of the
+path runs in the library's kernels - nothing is computed here.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+from typing import Optional
+
+import numpy as np
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libsam_b200.so"
+_lib = None
+
+SAM_K_MAX = 32
+SAM_MAX_SEPARATORS = 16
+
+_vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
+
+_SIGNATURES = {
+    "sam_build": (C.c_int, [_vp, _i64, _vp, _i32, C.POINTER(_vp)]),
+    "sam_sizes": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
+    "sam_export": (C.c_int, [_vp] * 7),
+    "sam_upload": (C.c_int, [_vp, _vp, _i64, _vp]),
+    "sam_free": (None, [_vp]),
+    "sam_workspace_bytes": (_i64, [_i32, _i32]),
+    "sam_workspace_init": (C.c_int, [_vp, _i64, _vp]),
+    "sam_draft": (C.c_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp]),
+    "sam_verify": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
+    "sam_step": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                           _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
+    "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                                _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_profile_enable": (C.c_int, [_i32]),
+    "sam_profile_count": (_i32, []),
+    "sam_profile_read": (C.c_int, [_i32, C.POINTER(C.c_float), C.POINTER(C.c_float)]),
+    "sam_strerror": (C.c_char_p, [C.c_int]),
+    "sam_last_cuda_error": (C.c_int, []),
+}
+
+
+class SamError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = sam_strerror(status)
+        if status == -4:
+            msg += f" (cudaError {sam_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    """Names every build of the library must export (those declared in include/sam.h)."""
+    return list(_SIGNATURES)
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2512_18337_b200.build` "
+                "(there is no CPU fallback)")
+        lib = C.CDLL(str(_LIB_PATH))
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _dev(t) -> Optional[int]:
+    """Device address of a torch tensor (must be contiguous, on CUDA) or a raw int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _host(a: Optional[np.ndarray], dtype) -> Optional[int]:
+    if a is None:
+        return None
+    if a.dtype != dtype or not a.flags.c_contiguous:
+        raise ValueError(f"expected a contiguous {np.dtype(dtype).name} array")
+    return a.ctypes.data
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise SamError(status, where)
+
+
+# ------------------------------------------------------------------ setup
+def sam_build(corpus: np.ndarray, separators) -> int:
+    """Host build; returns the opaque handle (release with sam_free)."""
+    corpus = np.ascontiguousarray(corpus, dtype=np.int32)
+    seps = np.ascontiguousarray(np.atleast_1d(separators), dtype=np.int32)
+    h = _vp()
+    _check(_load().sam_build(corpus.ctypes.data, corpus.shape[0], seps.ctypes.data if seps.size else None,
+                             seps.shape[0], C.byref(h)), "sam_build")
+    return h.value
+
+
+def sam_sizes(handle: int):
+    """(n_states, n_edges, device_bytes)."""
+    a, b, c = _i64(), _i64(), _i64()
+    _check(_load().sam_sizes(handle, C.byref(a), C.byref(b), C.byref(c)), "sam_sizes")
+    return a.value, b.value, c.value
+
+
+def sam_export(handle: int):
+    """Flat host arrays of the automaton as a dict of numpy arrays."""
+    S, E, _ = sam_sizes(handle)
+    out = dict(len=np.empty(S, np.int32), link=np.empty(S, np.int32), firstpos=np.empty(S, np.int32),
+               row_ptr=np.empty(S + 1, np.int64), edge_tok=np.empty(E, np.int32), edge_dst=np.empty(E, np.int32))
+    _check(_load().sam_export(handle, out["len"].ctypes.data, out["link"].ctypes.data,
+                              out["firstpos"].ctypes.data, out["row_ptr"].ctypes.data,
+                              out["edge_tok"].ctypes.data, out["edge_dst"].ctypes.data), "sam_export")
+    return out
+
+
+def sam_upload(handle: int, device_buf, nbytes: Optional[int] = None, stream=None) -> None:
+    nbytes = device_buf.numel() * device_buf.element_size() if nbytes is None else nbytes
+    _check(_load().sam_upload(handle, _dev(device_buf), nbytes, _stream(stream)), "sam_upload")
+
+
+def sam_free(handle: int) -> None:
+    _load().sam_free(handle)
+
+
+def sam_workspace_bytes(B: int, K: int) -> int:
+    n = _load().sam_workspace_bytes(B, K)
+    if n < 0:
+        raise SamError(int(n), "sam_workspace_bytes")
+    return int(n)
+
+
+def sam_workspace_init(workspace, nbytes: Optional[int] = None, stream=None) -> None:
+    nbytes = workspace.numel() * workspace.element_size() if nbytes is None else nbytes
+    _check(_load().sam_workspace_init(_dev(workspace), nbytes, _stream(stream)), "sam_workspace_init")
+
+
+# ------------------------------------------------------------------ hot path
+def sam_draft(handle, B, state, matched_len, new_tokens, ld, n_new, K, min_match, drafts, n_draft, stream=None):
+    _check(_load().sam_draft(handle, B, _dev(state), _dev(matched_len), _dev(new_tokens), ld, _dev(n_new),
+                             K, min_match, _dev(drafts), _dev(n_draft), _stream(stream)), "sam_draft")
+
+
+def sam_verify(logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+               workspace, workspace_bytes, stream=None):
+    _check(_load().sam_verify(_dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft), _dev(argmax_out),
+                              _dev(accepted), _dev(n_accepted), _dev(workspace), workspace_bytes,
+                              _stream(stream)), "sam_verify")
+
+
+def sam_step(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+             state, matched_len, min_match, next_drafts, next_n_draft, workspace, workspace_bytes, stream=None):
+    _check(_load().sam_step(handle, _dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft),
+                            _dev(argmax_out), _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len),
+                            min_match, _dev(next_drafts), _dev(next_n_draft), _dev(workspace), workspace_bytes,
+                            _stream(stream)), "sam_step")
+
+
+def _hostptr(a) -> Optional[int]:
+    """Host address of a numpy array or a CPU torch tensor (contiguous)."""
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        if not a.flags.c_contiguous:
+            raise ValueError("expected a contiguous array")
+        return a.ctypes.data
+    if a.is_cuda or not a.is_contiguous():
+        raise ValueError("expected a contiguous host tensor")
+    return a.data_ptr()
+
+
+def sam_step_host_staging_bytes(row_stride: int, B: int, K: int, V: int) -> int:
+    n = _load().sam_step_host_staging_bytes(row_stride, B, K, V)
+    if n < 0:
+        raise SamError(int(n), "sam_step_host_staging_bytes")
+    return int(n)
+
+
+def sam_step_host(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                  state, matched_len, min_match, next_drafts, next_n_draft, staging, staging_bytes, stream=None):
+    """All arrays are HOST memory (numpy or CPU torch tensors) except `staging` (device)."""
+    _check(_load().sam_step_host(handle, _hostptr(logits), row_stride, B, K, V, _hostptr(drafts), _hostptr(n_draft),
+                                 _hostptr(argmax_out), _hostptr(accepted), _hostptr(n_accepted), _hostptr(state),
+                                 _hostptr(matched_len), min_match, _hostptr(next_drafts), _hostptr(next_n_draft),
+                                 _dev(staging), staging_bytes, _stream(stream)), "sam_step_host")
+
+
+def sam_profile_enable(max_calls: int) -> None:
+    _check(_load().sam_profile_enable(max_calls), "sam_profile_enable")
+
+
+def sam_profile_count() -> int:
+    return int(_load().sam_profile_count())
+
+
+def sam_profile_read(call: int):
+    """(argmax_ms, accept_ms) of the call-th profiled sam_verify / sam_step."""
+    a, b = C.c_float(), C.c_float()
+    _check(_load().sam_profile_read(call, C.byref(a), C.byref(b)), "sam_profile_read")
+    return a.value, b.value
+
+
+def sam_strerror(status: int) -> str:
+    return _load().sam_strerror(status).decode()
+
+
+def sam_last_cuda_error() -> int:
+    return int(_load().sam_last_cuda_error())
+
+
+# ------------------------------------------------------------------ convenience holder
+class SamIndex:
+    """Owns a built handle and the torch tensor that holds its device blob (memory plumbing only)."""
+
+    def __init__(self, corpus: np.ndarray, separators, device="cuda:0", upload: bool = True):
+        self.handle = sam_build(corpus, separators)
+        self.n_states, self.n_edges, self.device_bytes = sam_sizes(self.handle)
+        self.blob = None
+        if upload:
+            import torch
+            self.blob = torch.empty(self.device_bytes, dtype=torch.uint8, device=device)
+            sam_upload(self.handle, self.blob)
+
+    def close(self):
+        h, self.handle = self.handle, None
+        if h:
+            sam_free(h)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,371 @@
+// C ABI of the library: argument checks, device-blob upload and kernel launches.
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sam.h"
+#include "sam_index.h"
+#include "sam_kernels.cuh"
+
+using namespace samb200;
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+inline int cuda_fail(cudaError_t e) {
+    g_last_cuda = static_cast<int>(e);
+    return SAM_ERR_CUDA;
+}
+
+#define SAM_CUDA(call)                                   \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) return cuda_fail(e__);   \
+    } while (0)
+
+struct DeviceInfo {
+    int sms = 0;
+};
+
+int device_info(DeviceInfo* out) {
+    static thread_local int cached_dev = -1;
+    static thread_local DeviceInfo cached;
+    int dev = 0;
+    SAM_CUDA(cudaGetDevice(&dev));
+    if (dev != cached_dev) {
+        int sms = 0;
+        SAM_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        cached.sms = sms;
+        cached_dev = dev;
+    }
+    *out = cached;
+    return SAM_OK;
+}
+
+// ---- optional per-kernel timing (events owned by the library) --------------------------------
+struct Profile {
+    std::vector<cudaEvent_t> ev;   // 3 per call
+    int32_t cap = 0, used = 0;
+};
+Profile g_prof;
+
+inline void prof_mark(int phase, cudaStream_t st) {
+    if (g_prof.used < g_prof.cap) cudaEventRecord(g_prof.ev[static_cast<size_t>(g_prof.used) * 3 + phase], st);
+}
+inline void prof_done() {
+    if (g_prof.used < g_prof.cap) ++g_prof.used;
+}
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_verify_args(const void* logits, int64_t stride, int32_t B, int32_t K, int32_t V,
+                      const int32_t* drafts, const int32_t* n_draft, int32_t* argmax_out,
+                      int32_t* accepted, int32_t* n_accepted, void* ws, int64_t ws_bytes) {
+    if (B < 0 || K < 1 || K > SAM_K_MAX || V < 1 || stride < V) return SAM_ERR_INVALID_ARG;
+    if (B == 0) return SAM_OK;
+    if (!logits || !drafts || !n_draft || !argmax_out || !accepted || !n_accepted || !ws) return SAM_ERR_INVALID_ARG;
+    if (!aligned(logits, 2) || !aligned(ws, 8)) return SAM_ERR_INVALID_ARG;
+    if (ws_bytes < sam_workspace_bytes(B, K)) return SAM_ERR_TOO_SMALL;
+    return SAM_OK;
+}
+
+int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
+                  cudaStream_t st) {
+    prof_mark(0, st);
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != SAM_OK) return rc;
+    const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
+    const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
+    const int64_t total = R * tiles_per_row;
+    int64_t grid = static_cast<int64_t>(di.sms) * 4;
+    if (grid > total) grid = total;
+    if (grid < 1) grid = 1;
+    argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys);
+    SAM_CUDA(cudaGetLastError());
+    prof_mark(1, st);
+    return SAM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sam_build(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep, sam_index** out) {
+    if (!corpus || !out || n < 1 || n > (int64_t(1) << 29)) return SAM_ERR_INVALID_ARG;
+    if (n_sep < 0 || n_sep > SAM_MAX_SEPARATORS || (n_sep > 0 && !separators)) return SAM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; ++i)
+        if (corpus[i] < 0 || corpus[i] >= (1 << 24)) return SAM_ERR_INVALID_ARG;
+    sam_index* idx = new (std::nothrow) sam_index();
+    if (!idx) return SAM_ERR_NOMEM;
+    const int rc = build_index(corpus, n, separators, n_sep, idx);
+    if (rc != SAM_OK) {
+        delete idx;
+        return rc;
+    }
+    *out = idx;
+    return SAM_OK;
+}
+
+int sam_sizes(const sam_index* idx, int64_t* n_states, int64_t* n_edges, int64_t* device_bytes) {
+    if (!idx) return SAM_ERR_INVALID_ARG;
+    if (n_states) *n_states = idx->layout.n_states;
+    if (n_edges) *n_edges = static_cast<int64_t>(idx->edge_tok.size());
+    if (device_bytes) *device_bytes = idx->layout.total;
+    return SAM_OK;
+}
+
+int sam_export(const sam_index* idx, int32_t* len, int32_t* link, int32_t* firstpos,
+               int64_t* row_ptr, int32_t* edge_tok, int32_t* edge_dst) {
+    if (!idx) return SAM_ERR_INVALID_ARG;
+    const size_t S = idx->len.size(), E = idx->edge_tok.size();
+    if (len) std::memcpy(len, idx->len.data(), S * 4);
+    if (link) std::memcpy(link, idx->link.data(), S * 4);
+    if (firstpos) std::memcpy(firstpos, idx->firstpos.data(), S * 4);
+    if (row_ptr) std::memcpy(row_ptr, idx->row_ptr.data(), (S + 1) * 8);
+    if (edge_tok) std::memcpy(edge_tok, idx->edge_tok.data(), E * 4);
+    if (edge_dst) std::memcpy(edge_dst, idx->edge_dst.data(), E * 4);
+    return SAM_OK;
+}
+
+int sam_upload(sam_index* idx, void* device_buf, int64_t bytes, void* cuda_stream) {
+    if (!idx || !device_buf || !aligned(device_buf, 256)) return SAM_ERR_INVALID_ARG;
+    const DeviceLayout& L = idx->layout;
+    if (bytes < L.total) return SAM_ERR_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    std::vector<StateRec> rec;
+    std::vector<Edge> wide;
+    std::vector<int32_t> root;
+    try {
+        rec.resize(static_cast<size_t>(L.n_states));
+        wide.resize(static_cast<size_t>(L.n_wide_edges));
+        root.resize(static_cast<size_t>(L.root_span));
+    } catch (const std::bad_alloc&) {
+        return SAM_ERR_NOMEM;
+    }
+    pack_records(*idx, rec.data(), wide.data(), root.data());
+    char* base = static_cast<char*>(device_buf);
+    SAM_CUDA(cudaMemcpyAsync(base + L.rec_off, rec.data(), rec.size() * sizeof(StateRec), cudaMemcpyHostToDevice, st));
+    if (!wide.empty())
+        SAM_CUDA(cudaMemcpyAsync(base + L.edge_off, wide.data(), wide.size() * sizeof(Edge), cudaMemcpyHostToDevice, st));
+    if (!root.empty())
+        SAM_CUDA(cudaMemcpyAsync(base + L.root_off, root.data(), root.size() * 4, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(base + L.corpus_off, idx->corpus.data(), idx->corpus.size() * 4, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaStreamSynchronize(st));
+    idx->device_buf = device_buf;
+    DeviceSam& d = idx->dev;
+    d.rec = reinterpret_cast<const StateRec*>(base + L.rec_off);
+    d.wide = reinterpret_cast<const Edge*>(base + L.edge_off);
+    d.root_dst = reinterpret_cast<const int32_t*>(base + L.root_off);
+    d.corpus = reinterpret_cast<const int32_t*>(base + L.corpus_off);
+    d.root_span = static_cast<int32_t>(L.root_span);
+    d.n_states = static_cast<int32_t>(L.n_states);
+    d.n_corpus = L.n_corpus;
+    d.n_sep = static_cast<int32_t>(idx->seps.size());
+    for (int k = 0; k < SAM_MAX_SEPARATORS; ++k) d.seps[k] = (k < d.n_sep) ? idx->seps[k] : -1;
+    return SAM_OK;
+}
+
+void sam_free(sam_index* idx) { delete idx; }
+
+int64_t sam_workspace_bytes(int32_t B, int32_t K) {
+    if (B < 0 || K < 1 || K > SAM_K_MAX) return SAM_ERR_INVALID_ARG;
+    const int64_t rows = static_cast<int64_t>(B) * (K + 1);
+    return ((rows * 8 + 255) / 256) * 256 + 256;
+}
+
+int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream) {
+    if (!workspace || bytes < 0 || !aligned(workspace, 8)) return SAM_ERR_INVALID_ARG;
+    SAM_CUDA(cudaMemsetAsync(workspace, 0, static_cast<size_t>(bytes), static_cast<cudaStream_t>(cuda_stream)));
+    return SAM_OK;
+}
+
+int sam_draft(const sam_index* idx, int32_t B, int32_t* state, int32_t* matched_len,
+              const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
+              int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, void* cuda_stream) {
+    if (!idx || B < 0 || K < 1 || K > SAM_K_MAX || min_match < 1 || ld < 0) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!state || !matched_len || !n_new || !drafts || !n_draft || (ld > 0 && !new_tokens)) return SAM_ERR_INVALID_ARG;
+    const int warps = 4;
+    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
+    draft_kernel<<<grid, warps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        idx->dev, B, state, matched_len, new_tokens, ld, n_new, K, min_match, drafts, n_draft);
+    SAM_CUDA(cudaGetLastError());
+    return SAM_OK;
+}
+
+int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+               const int32_t* drafts, const int32_t* n_draft,
+               int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+               void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
+                               n_accepted, workspace, workspace_bytes);
+    if (rc != SAM_OK || B == 0) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned long long* keys = static_cast<unsigned long long*>(workspace);
+    rc = launch_argmax(logits_bf16, row_stride_elems, static_cast<int64_t>(B) * (K + 1), V, keys, st);
+    if (rc != SAM_OK) return rc;
+    const int warps = 4;
+    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
+    accept_kernel<false><<<grid, warps * 32, 0, st>>>(
+        DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr);
+    SAM_CUDA(cudaGetLastError());
+    prof_mark(2, st);
+    prof_done();
+    return SAM_OK;
+}
+
+int sam_step(const sam_index* idx,
+             const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+             const int32_t* drafts, const int32_t* n_draft,
+             int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+             int32_t* state, int32_t* matched_len, int32_t min_match,
+             int32_t* next_drafts, int32_t* next_n_draft,
+             void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    if (!idx || min_match < 1) return SAM_ERR_INVALID_ARG;
+    int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
+                               n_accepted, workspace, workspace_bytes);
+    if (rc != SAM_OK) return rc;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!state || !matched_len || !next_drafts || !next_n_draft) return SAM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned long long* keys = static_cast<unsigned long long*>(workspace);
+    rc = launch_argmax(logits_bf16, row_stride_elems, static_cast<int64_t>(B) * (K + 1), V, keys, st);
+    if (rc != SAM_OK) return rc;
+    const int warps = 4;
+    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
+    accept_kernel<true><<<grid, warps * 32, 0, st>>>(
+        idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+        argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft);
+    SAM_CUDA(cudaGetLastError());
+    prof_mark(2, st);
+    prof_done();
+    return SAM_OK;
+}
+
+namespace {
+struct HostStepLayout {
+    int64_t logits, drafts, n_draft, argmax, accepted, n_accepted, state, mlen, ws, total;
+    int64_t logits_bytes, ws_bytes;
+};
+bool host_step_layout(int64_t stride, int32_t B, int32_t K, int32_t V, HostStepLayout* L) {
+    if (B < 0 || K < 1 || K > SAM_K_MAX || V < 1 || stride < V) return false;
+    auto up = [](int64_t x) { return (x + 255) & ~int64_t(255); };
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    L->logits_bytes = R > 0 ? ((R - 1) * stride + V) * 2 : 0;
+    L->ws_bytes = sam_workspace_bytes(B, K);
+    int64_t o = 0;
+    L->logits = o;     o = up(o + L->logits_bytes + 16);
+    L->drafts = o;     o = up(o + static_cast<int64_t>(B) * K * 4);
+    L->n_draft = o;    o = up(o + static_cast<int64_t>(B) * 4);
+    L->argmax = o;     o = up(o + R * 4);
+    L->accepted = o;   o = up(o + R * 4);
+    L->n_accepted = o; o = up(o + static_cast<int64_t>(B) * 4);
+    L->state = o;      o = up(o + static_cast<int64_t>(B) * 4);
+    L->mlen = o;       o = up(o + static_cast<int64_t>(B) * 4);
+    L->ws = o;         o = up(o + L->ws_bytes);
+    L->total = o;
+    return true;
+}
+}  // namespace
+
+int64_t sam_step_host_staging_bytes(int64_t row_stride_elems, int32_t B, int32_t K, int32_t V) {
+    HostStepLayout L;
+    if (!host_step_layout(row_stride_elems, B, K, V, &L)) return SAM_ERR_INVALID_ARG;
+    return L.total;
+}
+
+int sam_step_host(const sam_index* idx,
+                  const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                  const int32_t* drafts, const int32_t* n_draft,
+                  int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                  int32_t* state, int32_t* matched_len, int32_t min_match,
+                  int32_t* next_drafts, int32_t* next_n_draft,
+                  void* staging, int64_t staging_bytes, void* cuda_stream) {
+    HostStepLayout L;
+    if (!idx || !host_step_layout(row_stride_elems, B, K, V, &L) || min_match < 1) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!logits_bf16 || !drafts || !n_draft || !argmax_out || !accepted || !n_accepted || !state || !matched_len ||
+        !next_drafts || !next_n_draft || !staging || !aligned(staging, 256))
+        return SAM_ERR_INVALID_ARG;
+    if (staging_bytes < L.total) return SAM_ERR_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* d = static_cast<char*>(staging);
+    const size_t bB = static_cast<size_t>(B) * 4, bK = bB * K, bR = bB * (K + 1);
+    SAM_CUDA(cudaMemcpyAsync(d + L.logits, logits_bf16, static_cast<size_t>(L.logits_bytes), cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(d + L.drafts, drafts, bK, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(d + L.n_draft, n_draft, bB, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(d + L.state, state, bB, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(d + L.mlen, matched_len, bB, cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemsetAsync(d + L.ws, 0, static_cast<size_t>(L.ws_bytes), st));
+    int32_t* dd = reinterpret_cast<int32_t*>(d + L.drafts);
+    int32_t* dn = reinterpret_cast<int32_t*>(d + L.n_draft);
+    const int rc = sam_step(idx, d + L.logits, row_stride_elems, B, K, V, dd, dn,
+                            reinterpret_cast<int32_t*>(d + L.argmax), reinterpret_cast<int32_t*>(d + L.accepted),
+                            reinterpret_cast<int32_t*>(d + L.n_accepted), reinterpret_cast<int32_t*>(d + L.state),
+                            reinterpret_cast<int32_t*>(d + L.mlen), min_match, dd, dn, d + L.ws, L.ws_bytes, st);
+    if (rc != SAM_OK) return rc;
+    SAM_CUDA(cudaMemcpyAsync(argmax_out, d + L.argmax, bR, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(accepted, d + L.accepted, bR, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(n_accepted, d + L.n_accepted, bB, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(state, d + L.state, bB, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(matched_len, d + L.mlen, bB, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(next_drafts, d + L.drafts, bK, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaMemcpyAsync(next_n_draft, d + L.n_draft, bB, cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaStreamSynchronize(st));
+    return SAM_OK;
+}
+
+int sam_profile_enable(int32_t max_calls) {
+    if (max_calls < 0) return SAM_ERR_INVALID_ARG;
+    for (cudaEvent_t e : g_prof.ev) cudaEventDestroy(e);
+    g_prof.ev.clear();
+    g_prof.cap = g_prof.used = 0;
+    try {
+        g_prof.ev.reserve(static_cast<size_t>(max_calls) * 3);
+    } catch (const std::bad_alloc&) {
+        return SAM_ERR_NOMEM;
+    }
+    for (int64_t i = 0; i < static_cast<int64_t>(max_calls) * 3; ++i) {
+        cudaEvent_t e;
+        SAM_CUDA(cudaEventCreate(&e));
+        g_prof.ev.push_back(e);
+    }
+    g_prof.cap = max_calls;
+    return SAM_OK;
+}
+
+int32_t sam_profile_count(void) { return g_prof.used; }
+
+int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms) {
+    if (call < 0 || call >= g_prof.used) return SAM_ERR_INVALID_ARG;
+    const size_t o = static_cast<size_t>(call) * 3;
+    if (argmax_ms) SAM_CUDA(cudaEventElapsedTime(argmax_ms, g_prof.ev[o], g_prof.ev[o + 1]));
+    if (accept_ms) SAM_CUDA(cudaEventElapsedTime(accept_ms, g_prof.ev[o + 1], g_prof.ev[o + 2]));
+    return SAM_OK;
+}
+
+const char* sam_strerror(int status) {
+    switch (status) {
+        case SAM_OK: return "ok";
+        case SAM_ERR_INVALID_ARG: return "invalid argument";
+        case SAM_ERR_NOMEM: return "out of host memory";
+        case SAM_ERR_NOT_UPLOADED: return "automaton not uploaded to the device";
+        case SAM_ERR_CUDA: return "CUDA call failed";
+        case SAM_ERR_TOO_SMALL: return "caller buffer too small";
+        default: return "unknown status";
+    }
+}
+
+int sam_last_cuda_error(void) { return g_last_cuda; }
+
+}  // extern "C"

@@ -1,0 +1,396 @@
+// Device code of the draft + verify path (sm_100a). Included only by sam_capi.cu.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "sam_index.h"
+
+namespace samb200 {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+// ============================================================================================
+// Automaton walk and draft emission (Section 5.4.2; Algorithm 3 "FollowTransitions" / "Emit").
+// One warp per request stream; every lane holds the same (state, matched_len, record).
+// ============================================================================================
+
+struct RecRegs {
+    int4 a;  // len, link, firstpos, deg
+    int4 b;  // inline transitions / wide-row offset
+};
+
+__device__ __forceinline__ RecRegs load_rec(const DeviceSam& sam, int s) {
+    const int4* p = reinterpret_cast<const int4*>(sam.rec + s);
+    RecRegs r;
+    r.a = __ldg(p);
+    r.b = __ldg(p + 1);
+    return r;
+}
+
+__device__ __forceinline__ RecRegs root_rec() {
+    RecRegs r;
+    r.a = make_int4(0, -1, -1, 0);
+    r.b = make_int4(-1, -1, -1, -1);
+    return r;
+}
+
+// Warp-cooperative search of one ascending row of `deg` (tok, dst) pairs: 32-way narrowing
+// until at most 32 candidates remain, then one pass in which every lane compares its own entry.
+// Each round is one dependent memory access.
+__device__ __forceinline__ int row_search(const Edge* __restrict__ row, int deg, int c, int lane) {
+    int lo = 0, hi = deg;
+    while (hi - lo > 32) {
+        const int step = (hi - lo + 31) >> 5;
+        const int i = lo + lane * step;
+        const bool in = i < hi;
+        const int t = in ? __ldg(&row[i].tok) : 0;
+        const unsigned le = __ballot_sync(kFull, in && t <= c);
+        if (le == 0) return -1;             // c is below the first pivot of the range
+        const int k = __popc(le) - 1;       // pivots ascend, so `le` is a prefix mask
+        lo = lo + k * step;
+        hi = min(lo + step, hi);
+    }
+    const int i = lo + lane;
+    int2 e = make_int2(0, -1);
+    const bool in = i < hi;
+    if (in) e = __ldg(reinterpret_cast<const int2*>(row + i));
+    const unsigned hit = __ballot_sync(kFull, in && e.x == c);
+    if (hit == 0) return -1;
+    return __shfl_sync(kFull, e.y, __ffs(hit) - 1);
+}
+
+// Destination of the transition (s, c) or -1. `r` is the record of s.
+__device__ __forceinline__ int transition(const DeviceSam& sam, int s, const RecRegs& r, int c, int lane) {
+    if (s == 0) {
+        return (c >= 0 && c < sam.root_span) ? __ldg(sam.root_dst + c) : -1;
+    }
+    const int deg = r.a.w;
+    if (deg <= 2) {
+        if (deg >= 1 && r.b.x == c) return r.b.y;
+        if (deg == 2 && r.b.z == c) return r.b.w;
+        return -1;
+    }
+    return row_search(sam.wide + r.b.x, deg, c, lane);
+}
+
+// Consume one token: a transition extends the match by one; on a miss follow the suffix link
+// and shorten the match to that state's length; a miss at the root resets the match to zero.
+__device__ __forceinline__ void walk_token(const DeviceSam& sam, int c, int& s, int& L, RecRegs& r, int lane) {
+    for (;;) {
+        const int d = transition(sam, s, r, c, lane);
+        if (d >= 0) {
+            s = d;
+            L += 1;
+            r = load_rec(sam, s);
+            return;
+        }
+        if (s == 0) {
+            L = 0;
+            return;
+        }
+        s = r.a.y;
+        r = (s == 0) ? root_rec() : load_rec(sam, s);
+        L = r.a.x;
+    }
+}
+
+// A (state, matched_len) pair that this library did not produce is reset to the start pair
+// instead of being dereferenced.
+__device__ __forceinline__ void sanitize_stream_state(const DeviceSam& sam, int& s, int& L) {
+    if (s <= 0 || s >= sam.n_states || L < 0) {
+        s = 0;
+        L = 0;
+    }
+}
+
+__device__ __forceinline__ bool is_separator(const DeviceSam& sam, int tok) {
+    bool hit = false;
+#pragma unroll 1
+    for (int k = 0; k < sam.n_sep; ++k) hit |= (sam.seps[k] == tok);
+    return hit;
+}
+
+// Emit the continuation after the first occurrence of the matched suffix (K <= 32: one lane
+// per draft slot, one coalesced read of the corpus). Returns n_draft (same on every lane).
+__device__ __forceinline__ int emit_draft(const DeviceSam& sam, int L, const RecRegs& r, int K, int min_match,
+                                          int* __restrict__ drafts_row, int lane) {
+    int nd = 0;
+    int tok = -1;
+    if (L >= min_match) {                     // uniform across the warp
+        const int64_t pos = static_cast<int64_t>(r.a.z) + 1 + lane;
+        bool stop = true;
+        if (lane < K && pos < sam.n_corpus) {
+            tok = __ldg(sam.corpus + pos);
+            stop = is_separator(sam, tok);
+        }
+        const unsigned sm = __ballot_sync(kFull, stop);   // lanes >= K always stop
+        nd = __ffs(sm) - 1;                   // sm != 0 because K <= 32 and lane K.. stop (or nd = K)
+        if (sm == 0) nd = K;                  // K == 32 and nothing stopped
+        nd = min(nd, K);
+    }
+    if (lane < K) drafts_row[lane] = (lane < nd) ? tok : -1;
+    return nd;
+}
+
+// sam_draft: walk caller-provided tokens, then emit.
+__global__ void __launch_bounds__(128)
+draft_kernel(DeviceSam sam, int B, int* __restrict__ state, int* __restrict__ matched_len,
+             const int* __restrict__ new_tokens, int ld, const int* __restrict__ n_new,
+             int K, int min_match, int* __restrict__ drafts, int* __restrict__ n_draft) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= B) return;
+    int s = state[b];
+    int L = matched_len[b];
+    sanitize_stream_state(sam, s, L);
+    RecRegs r = (s == 0) ? root_rec() : load_rec(sam, s);
+    const int n = max(0, min(n_new[b], ld));
+    const int* row = new_tokens + static_cast<int64_t>(b) * ld;
+    for (int base = 0; base < n; base += 32) {
+        const int mine = (base + lane < n) ? __ldg(row + base + lane) : -1;
+        const int cnt = min(32, n - base);
+        for (int t = 0; t < cnt; ++t) {
+            const int c = __shfl_sync(kFull, mine, t);
+            walk_token(sam, c, s, L, r, lane);
+        }
+    }
+    const int nd = emit_draft(sam, L, r, K, min_match, drafts + static_cast<int64_t>(b) * K, lane);
+    if (lane == 0) {
+        state[b] = s;
+        matched_len[b] = L;
+        n_draft[b] = nd;
+    }
+}
+
+// ============================================================================================
+// Vocabulary argmax (Algorithm 3 "Validate with main LLM": the model's greedy choice per row).
+// Bandwidth-bound: every bf16 is read once. Ties go to the lowest index.
+// ============================================================================================
+
+// Monotone 16-bit key of a non-NaN bf16 value held in a float; -0 and +0 share a key; >= 1.
+__device__ __forceinline__ unsigned ordered_key(float x) {
+    unsigned b = __float_as_uint(x) >> 16;
+    if ((b & 0x7FFFu) == 0) b = 0;
+    return (b & 0x8000u) ? (~b & 0xFFFFu) : (b | 0x8000u);
+}
+
+// (value key, index) packed so that an unsigned 64-bit max picks the larger value and,
+// among equal values, the smaller index. Zero means "no candidate".
+__device__ __forceinline__ unsigned long long pack_candidate(float x, unsigned idx) {
+    return (static_cast<unsigned long long>(ordered_key(x)) << 32) | (0xFFFFFFFFu - idx);
+}
+
+__device__ __forceinline__ float bf16lo(unsigned u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(unsigned u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+__device__ __forceinline__ unsigned hmax2u(unsigned a, unsigned b) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
+    __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 m = __hmax2(x, y);        // a NaN operand is dropped, as in the scalar scan
+    return *reinterpret_cast<unsigned*>(&m);
+}
+
+// Maximum of the eight bf16 values of a 16-byte vector (NaN only if all eight are NaN).
+__device__ __forceinline__ float vec_max(const uint4& v) {
+    const unsigned m = hmax2u(hmax2u(v.x, v.y), hmax2u(v.z, v.w));
+    return fmaxf(bf16lo(m), bf16hi(m));
+}
+
+constexpr unsigned kNaN2 = 0x7FC07FC0u;
+
+// Replace the lanes of vector q that fall outside virtual elements [off, off + V) by NaN.
+__device__ __forceinline__ void mask_vector(uint4& v, long long q, int off, int V) {
+    unsigned w[4] = {v.x, v.y, v.z, v.w};
+    const long long e0 = q * 8;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const long long lo = e0 + 2 * k, hi = lo + 1;
+        if (lo < off || lo >= static_cast<long long>(off) + V) w[k] = (w[k] & 0xFFFF0000u) | 0x7FC0u;
+        if (hi < off || hi >= static_cast<long long>(off) + V) w[k] = (w[k] & 0x0000FFFFu) | 0x7FC00000u;
+    }
+    v = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// First position (0..7) in the vector whose value equals x; 8 if none.
+__device__ __forceinline__ int first_equal(const uint4& v, float x) {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    int e = 8;
+#pragma unroll
+    for (int k = 3; k >= 0; --k) {
+        if (bf16hi(w[k]) == x) e = 2 * k + 1;
+        if (bf16lo(w[k]) == x) e = 2 * k;
+    }
+    return e;
+}
+
+struct RowView {
+    const uint4* vec;   // 16-byte aligned start at or before the row's first element
+    int off;            // elements between vec and the row start (0..7)
+    int nvec;           // vectors covering the row
+};
+
+__device__ __forceinline__ RowView row_view(const __nv_bfloat16* logits, long long stride, long long row, int V) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(logits + row * stride);
+    const uintptr_t a0 = a & ~static_cast<uintptr_t>(15);
+    RowView rv;
+    rv.vec = reinterpret_cast<const uint4*>(a0);
+    rv.off = static_cast<int>((a - a0) >> 1);
+    rv.nvec = (rv.off + V + 7) >> 3;
+    return rv;
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+constexpr int kArgmaxThreads = 256;
+constexpr int kTileVec = 1024;    // 16-byte vectors per tile: 16 KB
+constexpr int kVecPerThread = kTileVec / kArgmaxThreads;
+
+// Turn a thread's (best value, vector index) into a packed candidate by re-reading that one
+// vector (an L2 hit: it was streamed moments ago) and locating the first equal element.
+__device__ __forceinline__ unsigned long long resolve_candidate(const RowView& rv, int V, float best, int bestq) {
+    if (bestq < 0) return 0ull;
+    uint4 v = __ldg(rv.vec + bestq);
+    if (bestq == 0 || bestq == rv.nvec - 1) mask_vector(v, bestq, rv.off, V);
+    const int e = first_equal(v, best);
+    const unsigned idx = static_cast<unsigned>(bestq * 8 + e - rv.off);
+    return pack_candidate(best, idx);
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(kFull, k, d);
+        k = (o > k) ? o : k;
+    }
+    return k;
+}
+
+// Generic streaming argmax: direct 16-byte global loads, any row alignment.
+// The R * tiles_per_row tiles are split into equal contiguous ranges, one per CTA; partial
+// results of a row meet in keys[row] through a 64-bit atomic max.
+__global__ void __launch_bounds__(kArgmaxThreads)
+argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
+                     int tiles_per_row, unsigned long long* __restrict__ keys) {
+    const long long total = R * tiles_per_row;
+    const long long t0 = total * blockIdx.x / gridDim.x;
+    const long long t1 = total * (blockIdx.x + 1) / gridDim.x;
+    const int lane = threadIdx.x & 31;
+    long long cur_row = -1;
+    RowView rv{};
+    float best = __int_as_float(0xff800000);   // -inf: only strictly greater values become candidates
+    int bestq = -1;
+
+    auto flush = [&]() {
+        if (cur_row < 0) return;
+        unsigned long long k = resolve_candidate(rv, V, best, bestq);
+        k = warp_max_u64(k);
+        if (lane == 0 && k != 0ull) atomicMax(keys + cur_row, k);
+    };
+
+    for (long long t = t0; t < t1; ++t) {
+        const long long row = t / tiles_per_row;
+        const int tile = static_cast<int>(t - row * tiles_per_row);
+        if (row != cur_row) {
+            flush();
+            cur_row = row;
+            rv = row_view(logits, stride, row, V);
+            best = __int_as_float(0xff800000);
+            bestq = -1;
+        }
+        const int q0 = tile * kTileVec + threadIdx.x;
+        uint4 v[kVecPerThread];
+#pragma unroll
+        for (int i = 0; i < kVecPerThread; ++i) {
+            const int q = q0 + i * kArgmaxThreads;
+            v[i] = make_uint4(kNaN2, kNaN2, kNaN2, kNaN2);
+            if (q < rv.nvec) v[i] = ld_stream(rv.vec + q);
+        }
+#pragma unroll
+        for (int i = 0; i < kVecPerThread; ++i) {
+            const int q = q0 + i * kArgmaxThreads;
+            if (q < rv.nvec) {
+                if (q == 0 || q == rv.nvec - 1) mask_vector(v[i], q, rv.off, V);
+                const float m = vec_max(v[i]);
+                if (m > best) { best = m; bestq = q; }
+            }
+        }
+    }
+    flush();
+}
+
+// ============================================================================================
+// Accept + feedback (Algorithm 3: commit the matched prefix, fall back to the model's token at
+// the first mismatch, then follow the automaton over what was committed and draft again).
+// One warp per stream. Also decodes the packed argmax candidates and re-zeroes them.
+// ============================================================================================
+template <bool kWalk>
+__global__ void __launch_bounds__(128)
+accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long stride, int B, int K,
+              const int* __restrict__ drafts, const int* __restrict__ n_draft,
+              int* __restrict__ argmax_out, int* __restrict__ accepted, int* __restrict__ n_accepted,
+              unsigned long long* __restrict__ keys,
+              int* __restrict__ state, int* __restrict__ matched_len, int min_match,
+              int* __restrict__ next_drafts, int* __restrict__ next_n_draft) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const int K1 = K + 1;
+    const long long row0 = static_cast<long long>(b) * K1;
+
+    // rows j = lane and j = lane + 32 (K + 1 <= 33)
+    int am[2] = {-1, -1};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int j = lane + 32 * h;
+        if (j < K1) {
+            const unsigned long long k = keys[row0 + j];
+            keys[row0 + j] = 0ull;
+            int idx = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
+            const unsigned short x0 = __ldg(reinterpret_cast<const unsigned short*>(logits + (row0 + j) * stride));
+            if ((x0 & 0x7FFFu) > 0x7F80u) idx = 0;     // element 0 is NaN: nothing ever compares greater
+            am[h] = idx;
+            argmax_out[row0 + j] = idx;
+        }
+    }
+
+    const int nd = max(0, min(n_draft[b], K));
+    const int d = (lane < K) ? drafts[static_cast<long long>(b) * K + lane] : -1;
+    const unsigned mism = __ballot_sync(kFull, lane < nd && d != am[0]);
+    const int a = mism ? (__ffs(mism) - 1) : nd;        // accepted draft tokens
+    const int bonus_lo = __shfl_sync(kFull, am[0], a & 31);
+    const int bonus_hi = __shfl_sync(kFull, am[1], 0);
+    const int bonus = (a < 32) ? bonus_lo : bonus_hi;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int j = lane + 32 * h;
+        if (j < K1) accepted[row0 + j] = (j < a) ? d : ((j == a) ? bonus : -1);
+    }
+    if (lane == 0) n_accepted[b] = a + 1;
+
+    if (kWalk) {
+        int s = state[b];
+        int L = matched_len[b];
+        sanitize_stream_state(sam, s, L);
+        RecRegs r = (s == 0) ? root_rec() : load_rec(sam, s);
+        for (int t = 0; t < a; ++t) {
+            const int c = __shfl_sync(kFull, d, t);
+            walk_token(sam, c, s, L, r, lane);
+        }
+        walk_token(sam, bonus, s, L, r, lane);
+        const int nn = emit_draft(sam, L, r, K, min_match, next_drafts + static_cast<long long>(b) * K, lane);
+        if (lane == 0) {
+            state[b] = s;
+            matched_len[b] = L;
+            next_n_draft[b] = nn;
+        }
+    }
+}
+
+}  // namespace samb200

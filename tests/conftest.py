@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The CUDA library is built in-tree (nvcc cross-compiles without a GPU) before any test."""
+    from paper_2512_18337_b200.build import build
+    build()
+
+
 def pytest_collection_modifyitems(config, items):
     """GPU tests are skipped, not failed, when no device is present."""
     try:
