@@ -40,6 +40,8 @@ extern "C" {
 #define SAM_ERR_CUDA          (-4)  /* a CUDA runtime call or kernel launch failed; see sam_last_cuda_error */
 #define SAM_ERR_TOO_SMALL     (-5)  /* caller buffer (device blob, workspace) smaller than required */
 
+#define SAM_ERR_TOO_LARGE     (-6)  /* size beyond a built-in limit of the called entry point */
+
 #define SAM_K_MAX             32    /* largest draft length K accepted by the hot path */
 #define SAM_MAX_SEPARATORS    16    /* largest number of separator ids */
 
@@ -147,6 +149,32 @@ int sam_step(const sam_index* idx,
              int32_t* state, int32_t* matched_len, int32_t min_match,
              int32_t* next_drafts, int32_t* next_n_draft,
              void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* Allocation-free form of sam_verify (a packaging variant; the paper has no counterpart).
+ * Some callers cannot obtain device scratch at all: a plugin running inside a serving engine
+ * that has already handed every free byte of device memory to its own pools (a late cudaMalloc
+ * there fails, or stalls the whole device while it runs), or a caller that only holds raw
+ * pointers from another runtime and has no allocator to ask.  For them the per-row scratch of
+ * the verification kernels lives inside the library image itself, in a fixed device array of
+ * SAM_STATIC_MAX_ROWS 64-bit words (128 KiB) that every GPU which loads the library holds until
+ * the process exits.  Arguments, results and semantics are exactly those of sam_verify, minus
+ * the workspace; inputs and outputs are still the caller's device buffers.
+ *   - B * (K + 1) must not exceed SAM_STATIC_MAX_ROWS, otherwise SAM_ERR_TOO_LARGE is returned
+ *     and nothing is launched.
+ *   - The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library
+ *     routine): it zero-fills the rows it is about to use with a stream-ordered memset and
+ *     enqueues the two kernels.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current) and keeps it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left
+ *     in it: two calls that overlap on the GPU (different streams, no ordering between them)
+ *     race on it and return garbage.  Order them, or use sam_verify with separate workspaces.
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_LARGE, SAM_ERR_CUDA. */
+#define SAM_STATIC_MAX_ROWS   16384
+int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                      const int32_t* drafts, const int32_t* n_draft,
+                      int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                      void* cuda_stream);
 
 /* Host-buffer form of sam_step, for callers whose logits and bookkeeping live in host memory
  * (Algorithm 3, one loop iteration, end to end).  Copies logits [B*(K+1) rows, row_stride_elems

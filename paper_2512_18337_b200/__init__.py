@@ -24,6 +24,7 @@ from .binding import (  # noqa: F401
     sam_strerror,
     sam_upload,
     sam_verify,
+    sam_verify_static,
     sam_workspace_bytes,
     sam_workspace_init,
 )

@@ -18,6 +18,7 @@ _lib = None
 
 SAM_K_MAX = 32
 SAM_MAX_SEPARATORS = 16
+SAM_STATIC_MAX_ROWS = 16384
 
 _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 
@@ -33,6 +34,7 @@ _SIGNATURES = {
     "sam_verify": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
     "sam_step": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                            _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_verify_static": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
@@ -174,6 +176,16 @@ def sam_verify(logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepte
     _check(_load().sam_verify(_dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft), _dev(argmax_out),
                               _dev(accepted), _dev(n_accepted), _dev(workspace), workspace_bytes,
                               _stream(stream)), "sam_verify")
+
+
+def sam_verify_static(logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted, stream=None):
+    """sam_verify for callers that cannot allocate device scratch (an engine plugin whose host has
+    already claimed all device memory, or code that only holds foreign raw pointers): the scratch is
+    a fixed array inside the library, so B*(K+1) <= SAM_STATIC_MAX_ROWS and calls on one GPU must
+    not overlap.  Same outputs as sam_verify."""
+    _check(_load().sam_verify_static(_dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft),
+                                     _dev(argmax_out), _dev(accepted), _dev(n_accepted), _stream(stream)),
+           "sam_verify_static")
 
 
 def sam_step(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,

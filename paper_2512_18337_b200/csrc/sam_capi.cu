@@ -3,6 +3,7 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -277,6 +278,61 @@ bool host_step_layout(int64_t stride, int32_t B, int32_t K, int32_t V, HostStepL
 }
 }  // namespace
 
+// ---- allocation-free verification ------------------------------------------------------------
+// The scratch words live in the library image: one array per GPU that loads the module, zero at
+// load time, shared by every sam_verify_static call on that GPU.
+static __device__ __align__(256) unsigned long long g_static_keys[SAM_STATIC_MAX_ROWS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+unsigned long long* g_static_keys_addr[kMaxDevices] = {};   // device address of g_static_keys, per device
+
+// In host code `g_static_keys` is only a handle for the runtime, not an address a kernel can use:
+// the real device address is looked up once per device, with that device current.
+int static_scratch(unsigned long long** out) {
+    int dev = -1;
+    SAM_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SAM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_keys_addr[dev]) {
+        unsigned long long* ptr = nullptr;
+        SAM_CUDA(cudaGetSymbolAddress((void**)&ptr, g_static_keys));
+        g_static_keys_addr[dev] = ptr;
+    }
+    *out = g_static_keys_addr[dev];
+    return SAM_OK;
+}
+}  // namespace
+
+int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                      const int32_t* drafts, const int32_t* n_draft,
+                      int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted, void* cuda_stream) {
+    if (B < 0 || K < 1 || K > SAM_K_MAX) return SAM_ERR_INVALID_ARG;
+    const int64_t rows = static_cast<int64_t>(B) * (K + 1);
+    if (rows > SAM_STATIC_MAX_ROWS) return SAM_ERR_TOO_LARGE;
+    unsigned long long* keys = nullptr;
+    int rc = static_scratch(&keys);
+    if (rc != SAM_OK) return rc;
+    rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
+                           n_accepted, keys, static_cast<int64_t>(SAM_STATIC_MAX_ROWS) * 8 + 512);
+    if (rc != SAM_OK || B == 0) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // whatever an earlier (possibly failed) call left behind, these rows start from zero
+    SAM_CUDA(cudaMemsetAsync(keys, 0, static_cast<size_t>(rows) * 8, st));
+    rc = launch_argmax(logits_bf16, row_stride_elems, rows, V, keys, st);
+    if (rc != SAM_OK) return rc;
+    const int warps = 4;
+    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
+    accept_kernel<false><<<grid, warps * 32, 0, st>>>(
+        DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr);
+    SAM_CUDA(cudaGetLastError());
+    prof_mark(2, st);
+    prof_done();
+    return SAM_OK;
+}
+
 int64_t sam_step_host_staging_bytes(int64_t row_stride_elems, int32_t B, int32_t K, int32_t V) {
     HostStepLayout L;
     if (!host_step_layout(row_stride_elems, B, K, V, &L)) return SAM_ERR_INVALID_ARG;
@@ -362,6 +418,7 @@ const char* sam_strerror(int status) {
         case SAM_ERR_NOT_UPLOADED: return "automaton not uploaded to the device";
         case SAM_ERR_CUDA: return "CUDA call failed";
         case SAM_ERR_TOO_SMALL: return "caller buffer too small";
+        case SAM_ERR_TOO_LARGE: return "size exceeds a built-in limit of this entry point";
         default: return "unknown status";
     }
 }
