@@ -96,6 +96,13 @@ int64_t sam_workspace_bytes(int32_t B, int32_t K);
  * must not overlap on the device. */
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
 
+/* Reads the status word the verification kernels keep at the end of the scratch: 0 = fine,
+ * 1 = a kernel gave up on one of its internal (bounded) waits and the outputs of that call are
+ * not valid - re-initialise the scratch and retry.  Copies one int to the host and synchronises
+ * the stream: a diagnostic, not a hot-path call.  B and K locate the word (same values as in
+ * the calls that used the scratch). */
+int sam_workspace_status(const void* workspace, int32_t B, int32_t K, int32_t* status_out, void* cuda_stream);
+
 /* ---------------------------------------------------------------- hot path (device, async) */
 
 /* Draft (Section 5.4.2; Algorithm 3 "FollowTransitions" and "Emit speculative tokens").
@@ -204,6 +211,10 @@ int sam_step_host(const sam_index* idx,
  * milliseconds; the stream must have been synchronised by the caller first.
  * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
 int sam_profile_enable(int32_t max_calls);
+/* Selects the argmax kernel for later calls (process-wide; for measurements and tests):
+ * 0 = by alignment (default: bulk-copy pipeline when the logits base and row stride are 16-byte
+ * aligned, direct loads otherwise), 1 = always direct loads, 2 = same as 0. */
+int sam_set_argmax_variant(int32_t variant);
 int32_t sam_profile_count(void);
 int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms);
 

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     sam_profile_count,
     sam_profile_enable,
     sam_profile_read,
+    sam_set_argmax_variant,
     sam_sizes,
     sam_step,
     sam_step_host,
@@ -27,4 +28,5 @@ from .binding import (  # noqa: F401
     sam_verify_static,
     sam_workspace_bytes,
     sam_workspace_init,
+    sam_workspace_status,
 )

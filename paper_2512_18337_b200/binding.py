@@ -12,8 +12,11 @@ from typing import Optional
 
 import numpy as np
 
+import os
+
 _PKG = Path(__file__).resolve().parent
-_LIB_PATH = _PKG / "libsam_b200.so"
+# SAM_B200_LIB lets a tuning run point at another build of this same library
+_LIB_PATH = Path(os.environ.get("SAM_B200_LIB", _PKG / "libsam_b200.so"))
 _lib = None
 
 SAM_K_MAX = 32
@@ -38,6 +41,8 @@ _SIGNATURES = {
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_workspace_status": (C.c_int, [_vp, _i32, _i32, C.POINTER(_i32), _vp]),
+    "sam_set_argmax_variant": (C.c_int, [_i32]),
     "sam_profile_enable": (C.c_int, [_i32]),
     "sam_profile_count": (_i32, []),
     "sam_profile_read": (C.c_int, [_i32, C.POINTER(C.c_float), C.POINTER(C.c_float)]),
@@ -223,6 +228,16 @@ def sam_step_host(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_o
                                  _hostptr(argmax_out), _hostptr(accepted), _hostptr(n_accepted), _hostptr(state),
                                  _hostptr(matched_len), min_match, _hostptr(next_drafts), _hostptr(next_n_draft),
                                  _dev(staging), staging_bytes, _stream(stream)), "sam_step_host")
+
+
+def sam_workspace_status(workspace, B: int, K: int, stream=None) -> int:
+    out = _i32(0)
+    _check(_load().sam_workspace_status(_dev(workspace), B, K, C.byref(out), _stream(stream)), "sam_workspace_status")
+    return int(out.value)
+
+
+def sam_set_argmax_variant(variant: int) -> None:
+    _check(_load().sam_set_argmax_variant(variant), "sam_set_argmax_variant")
 
 
 def sam_profile_enable(max_calls: int) -> None:

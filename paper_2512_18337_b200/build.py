@@ -10,7 +10,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libsam_b200.so"
 SOURCES = [CSRC / "sam_capi.cu", CSRC / "sam_build.cpp"]
-HEADERS = [ROOT / "include" / "sam.h", CSRC / "sam_index.h", CSRC / "sam_kernels.cuh"]
+HEADERS = [ROOT / "include" / "sam.h", CSRC / "sam_index.h", CSRC / "sam_kernels.cuh", CSRC / "argmax_bulk.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -10,6 +10,7 @@
 #include "sam.h"
 #include "sam_index.h"
 #include "sam_kernels.cuh"
+#include "argmax_bulk.cuh"
 
 using namespace samb200;
 
@@ -74,20 +75,50 @@ int check_verify_args(const void* logits, int64_t stride, int32_t B, int32_t K, 
     return SAM_OK;
 }
 
+int g_argmax_variant = 0;   // 0 = choose by alignment, 1 = direct loads, 2 = bulk-copy pipeline (if alignment allows)
+
+inline int* status_word(unsigned long long* keys, int64_t R) {
+    return reinterpret_cast<int*>(reinterpret_cast<char*>(keys) + ((R * 8 + 255) / 256) * 256);
+}
+
+// Enqueues the argmax over R rows; partial results land in keys[R], `status` receives a non-zero
+// code if a kernel gives up on an internal wait.
 int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
-                  cudaStream_t st) {
+                  int* status, cudaStream_t st) {
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != SAM_OK) return rc;
-    const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
-    const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
-    const int64_t total = R * tiles_per_row;
-    int64_t grid = static_cast<int64_t>(di.sms) * 4;
-    if (grid > total) grid = total;
-    if (grid < 1) grid = 1;
-    argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys);
+    const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0;
+    const bool bulk = rows_aligned && g_argmax_variant != 1;
+    if (bulk) {
+        static thread_local int attr_dev = -1;
+        int dev = 0;
+        SAM_CUDA(cudaGetDevice(&dev));
+        if (attr_dev != dev) {
+            SAM_CUDA(cudaFuncSetAttribute(argmax_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kBulkSmemBytes)));
+            attr_dev = dev;
+        }
+        const int64_t nvec = V / 8;
+        const int tiles_per_row = static_cast<int>(nvec > 0 ? (nvec + kBulkTileVec - 1) / kBulkTileVec : 1);
+        const int tile_vec = static_cast<int>(nvec > 0 ? (nvec + tiles_per_row - 1) / tiles_per_row : 1);
+        const int64_t total = R * tiles_per_row;
+        int64_t grid = di.sms;
+        if (grid > total) grid = total;
+        if (grid < 1) grid = 1;
+        argmax_bulk_kernel<<<static_cast<unsigned>(grid), kBulkThreads, kBulkSmemBytes, st>>>(
+            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status);
+    } else {
+        const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
+        const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
+        const int64_t total = R * tiles_per_row;
+        int64_t grid = static_cast<int64_t>(di.sms) * 4;
+        if (grid > total) grid = total;
+        if (grid < 1) grid = 1;
+        argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys);
+    }
     SAM_CUDA(cudaGetLastError());
     prof_mark(1, st);
     return SAM_OK;
@@ -210,7 +241,8 @@ int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int
     if (rc != SAM_OK || B == 0) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     unsigned long long* keys = static_cast<unsigned long long*>(workspace);
-    rc = launch_argmax(logits_bf16, row_stride_elems, static_cast<int64_t>(B) * (K + 1), V, keys, st);
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, status_word(keys, R), st);
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
@@ -239,7 +271,8 @@ int sam_step(const sam_index* idx,
     if (!state || !matched_len || !next_drafts || !next_n_draft) return SAM_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     unsigned long long* keys = static_cast<unsigned long long*>(workspace);
-    rc = launch_argmax(logits_bf16, row_stride_elems, static_cast<int64_t>(B) * (K + 1), V, keys, st);
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, status_word(keys, R), st);
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
@@ -281,7 +314,7 @@ bool host_step_layout(int64_t stride, int32_t B, int32_t K, int32_t V, HostStepL
 // ---- allocation-free verification ------------------------------------------------------------
 // The scratch words live in the library image: one array per GPU that loads the module, zero at
 // load time, shared by every sam_verify_static call on that GPU.
-static __device__ __align__(256) unsigned long long g_static_keys[SAM_STATIC_MAX_ROWS];
+static __device__ __align__(256) unsigned long long g_static_keys[SAM_STATIC_MAX_ROWS + 32];   // + status word
 
 namespace {
 constexpr int kMaxDevices = 64;
@@ -320,7 +353,8 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // whatever an earlier (possibly failed) call left behind, these rows start from zero
     SAM_CUDA(cudaMemsetAsync(keys, 0, static_cast<size_t>(rows) * 8, st));
-    rc = launch_argmax(logits_bf16, row_stride_elems, rows, V, keys, st);
+    rc = launch_argmax(logits_bf16, row_stride_elems, rows, V, keys,
+                       reinterpret_cast<int*>(keys + SAM_STATIC_MAX_ROWS), st);
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
@@ -407,6 +441,22 @@ int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms) {
     const size_t o = static_cast<size_t>(call) * 3;
     if (argmax_ms) SAM_CUDA(cudaEventElapsedTime(argmax_ms, g_prof.ev[o], g_prof.ev[o + 1]));
     if (accept_ms) SAM_CUDA(cudaEventElapsedTime(accept_ms, g_prof.ev[o + 1], g_prof.ev[o + 2]));
+    return SAM_OK;
+}
+
+int sam_workspace_status(const void* workspace, int32_t B, int32_t K, int32_t* status_out, void* cuda_stream) {
+    if (!workspace || !status_out || B < 0 || K < 1 || K > SAM_K_MAX) return SAM_ERR_INVALID_ARG;
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    const int* w = status_word(static_cast<unsigned long long*>(const_cast<void*>(workspace)), R);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SAM_CUDA(cudaMemcpyAsync(status_out, w, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaStreamSynchronize(st));
+    return SAM_OK;
+}
+
+int sam_set_argmax_variant(int32_t variant) {
+    if (variant < 0 || variant > 2) return SAM_ERR_INVALID_ARG;
+    g_argmax_variant = variant;
     return SAM_OK;
 }
 

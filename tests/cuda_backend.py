@@ -64,6 +64,9 @@ class CudaBackend:
                    self.argmax, self.accepted, self.n_accepted, self.state, self.mlen, c.min_match,
                    self.drafts, self.n_draft, self.ws, self.ws_bytes)
 
+    def status(self) -> int:
+        return S.sam_workspace_status(self.ws, self.cfg.B, self.cfg.K)
+
     def step(self, drafts, n_draft):
         # the device already holds drafts/n_draft from the previous call; the arguments are the host copies
         self.launch_step()

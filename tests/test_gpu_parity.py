@@ -21,7 +21,7 @@ def _i32(x):
     return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(DEV)
 
 
-def _verify_gpu(bits: np.ndarray, V, B, K, drafts, n_draft, dev_tensor=None):
+def _verify_gpu(bits: np.ndarray, V, B, K, drafts, n_draft, dev_tensor=None, variant=0):
     """bits: [B*(K+1), stride] uint16 host. Returns argmax, accepted, n_accepted (numpy)."""
     lg = bits_to_device(bits) if dev_tensor is None else dev_tensor
     stride = bits.shape[1]
@@ -32,9 +32,14 @@ def _verify_gpu(bits: np.ndarray, V, B, K, drafts, n_draft, dev_tensor=None):
     ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
     S.sam_workspace_init(ws, wsb)
     d, nd = _i32(drafts), _i32(n_draft)
-    for _ in range(2):   # twice: the scratch must come back zeroed
-        S.sam_verify(lg, stride, B, K, V, d, nd, am, acc, nacc, ws, wsb)
-    torch.cuda.synchronize()
+    S.sam_set_argmax_variant(variant)
+    try:
+        for _ in range(2):   # twice: the scratch must come back zeroed
+            S.sam_verify(lg, stride, B, K, V, d, nd, am, acc, nacc, ws, wsb)
+        torch.cuda.synchronize()
+    finally:
+        S.sam_set_argmax_variant(0)
+    assert S.sam_workspace_status(ws, B, K) == 0
     assert int(ws.to(torch.int32).abs().sum()) == 0
     return am.cpu().numpy(), acc.cpu().numpy(), nacc.cpu().numpy()
 
@@ -48,15 +53,17 @@ def _check_verify(bits, V, B, K, rng):
         keep = rng.random(nd) < 0.8
         drafts[b, :nd] = np.where(keep, am_o[b, :nd], rng.integers(0, V, size=nd))
     acc_o, nacc_o = oracle.accept_batch(drafts, n_draft, am_o)
-    am, acc, nacc = _verify_gpu(bits, V, B, K, drafts, n_draft)
-    assert (am == am_o).all()
-    assert (nacc == nacc_o).all() and (acc == acc_o).all()
+    for variant in (0, 1):     # 0: bulk-copy pipeline when rows are 16-byte aligned; 1: direct loads always
+        am, acc, nacc = _verify_gpu(bits, V, B, K, drafts, n_draft, variant=variant)
+        assert (am == am_o).all(), variant
+        assert (nacc == nacc_o).all() and (acc == acc_o).all(), variant
 
 
 @pytest.mark.parametrize("V,pad,B,K", [
     (1, 0, 3, 1), (7, 0, 3, 2), (8, 0, 2, 3), (9, 7, 5, 4), (1000, 0, 4, 8), (1000, 3, 4, 8),
     (4097, 0, 6, 5), (4097, 8, 6, 5), (50257, 0, 3, 7), (50257, 1, 3, 7), (151936, 0, 2, 8),
-    (151936, 8, 3, 32), (8192 * 3, 0, 40, 16), (8191, 1, 33, 31),
+    (151936, 8, 3, 32), (8192 * 3, 0, 40, 16), (8191, 1, 33, 31), (8192 * 13 + 24, 0, 7, 3), (8192 * 12, 8, 9, 2),
+    (3, 5, 300, 1), (8200, 0, 1, 1), (8192 * 25 + 5, 3, 2, 2), (32768 * 3, 0, 5, 2), (32768 * 2 + 8, 0, 4, 1), (32768 * 2 - 3, 3, 4, 1),
 ])
 def test_verify_parity_shapes(V, pad, B, K):
     """Row lengths around vector/tile edges, misaligned row strides, every K edge."""
