@@ -34,7 +34,8 @@ constexpr int kBulkTileBytes = kBulkTileVec * 16;
 constexpr int kBulkStages = SAM_BULK_STAGES;           // ring of kBulkStages * kBulkTileBytes (<= ~200 KB)
 constexpr int kBulkConsumerWarps = SAM_BULK_CONSUMER_WARPS;
 constexpr int kBulkConsumers = kBulkConsumerWarps * 32;
-constexpr int kBulkThreads = kBulkConsumers + 32;      // + one producer warp
+constexpr int kBulkWalkerWarps = 2;                    // spare warps that walk ahead along the drafts
+constexpr int kBulkThreads = kBulkConsumers + 32 + kBulkWalkerWarps * 32;   // consumers, producer warp, walkers
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr size_t kBulkSmemBytes = static_cast<size_t>(kBulkStages) * kBulkTileBytes + 1024;
 
@@ -93,7 +94,7 @@ struct BulkShared {
 __global__ void __launch_bounds__(kBulkThreads, 1)
 argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
                    int tiles_per_row, int tile_vec, unsigned long long* __restrict__ keys,
-                   int* __restrict__ status) {
+                   int* __restrict__ status, DeviceSam sam, PreWalk pw) {
     // tile_vec <= kBulkTileVec: vectors per tile, chosen by the host so that a row splits into
     // tiles_per_row nearly equal tiles (large tiles amortise the per-tile hand-shake best).
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -150,6 +151,13 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                 *abort = 1;
                 atomicExch(status, kStatusWaitTimeout);
             }
+        }
+    } else if (warp > kBulkConsumerWarps) {
+        // ------------------------------------------------------------------ walk-ahead warps
+        if (pw.enabled) {
+            const int w = warp - kBulkConsumerWarps - 1;
+            for (int b = blockIdx.x * kBulkWalkerWarps + w; b < pw.B; b += gridDim.x * kBulkWalkerWarps)
+                prewalk_stream(sam, pw, b, lane);
         }
     } else {
         // ------------------------------------------------------------------ consumers

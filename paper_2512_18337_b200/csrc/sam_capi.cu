@@ -1,6 +1,7 @@
 // C ABI of the library: argument checks, device-blob upload and kernel launches.
 #include <cuda_runtime.h>
 
+#include <cstdint>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -81,10 +82,35 @@ inline int* status_word(unsigned long long* keys, int64_t R) {
     return reinterpret_cast<int*>(reinterpret_cast<char*>(keys) + ((R * 8 + 255) / 256) * 256);
 }
 
-// Enqueues the argmax over R rows; partial results land in keys[R], `status` receives a non-zero
-// code if a kernel gives up on an internal wait.
+// Partial results land in keys[R]; `status` receives a non-zero code if a kernel gives up on an
+// internal wait.
+// Layout of the verification scratch: keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K]
+struct Scratch {
+    unsigned long long* keys;
+    int* status;
+    int* pre_state;
+    int* pre_len;
+    int64_t bytes;
+};
+Scratch scratch_layout(void* base, int32_t B, int32_t K) {
+    auto up = [](int64_t x) { return (x + 255) & ~int64_t(255); };
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    char* p = static_cast<char*>(base);
+    Scratch s;
+    int64_t o = 0;
+    s.keys = reinterpret_cast<unsigned long long*>(p + o);  o = up(o + R * 8);
+    s.status = reinterpret_cast<int*>(p + o);               o += 256;
+    s.pre_state = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * K * 4);
+    s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * K * 4);
+    s.bytes = o;
+    return s;
+}
+
+// Enqueues the argmax over R rows (and, when pw.enabled and the bulk kernel runs, the walk-ahead
+// along the drafts).  *did_prewalk tells the caller whether pre_state / pre_len will be filled.
 int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
-                  int* status, cudaStream_t st) {
+                  int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
+                  bool* did_prewalk = nullptr) {
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);
@@ -108,7 +134,9 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid > total) grid = total;
         if (grid < 1) grid = 1;
         argmax_bulk_kernel<<<static_cast<unsigned>(grid), kBulkThreads, kBulkSmemBytes, st>>>(
-            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status);
+            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status,
+            sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{});
+        if (did_prewalk) *did_prewalk = (pw != nullptr && pw->enabled != 0);
     } else {
         const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
         const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
@@ -207,8 +235,7 @@ void sam_free(sam_index* idx) { delete idx; }
 
 int64_t sam_workspace_bytes(int32_t B, int32_t K) {
     if (B < 0 || K < 1 || K > SAM_K_MAX) return SAM_ERR_INVALID_ARG;
-    const int64_t rows = static_cast<int64_t>(B) * (K + 1);
-    return ((rows * 8 + 255) / 256) * 256 + 256;
+    return scratch_layout(nullptr, B, K).bytes;
 }
 
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream) {
@@ -246,9 +273,9 @@ int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    accept_kernel<false><<<grid, warps * 32, 0, st>>>(
+    accept_kernel<kTailVerifyOnly><<<grid, warps * 32, 0, st>>>(
         DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr);
+        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr, nullptr, nullptr);
     SAM_CUDA(cudaGetLastError());
     prof_mark(2, st);
     prof_done();
@@ -272,13 +299,24 @@ int sam_step(const sam_index* idx,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     unsigned long long* keys = static_cast<unsigned long long*>(workspace);
     const int64_t R = static_cast<int64_t>(B) * (K + 1);
-    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, status_word(keys, R), st);
+    const Scratch sc = scratch_layout(workspace, B, K);
+    PreWalk pw{state, matched_len, drafts, n_draft, sc.pre_state, sc.pre_len, B, K, 1};
+    bool did_prewalk = false;
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, sc.status, st, &idx->dev, &pw, &did_prewalk);
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    accept_kernel<true><<<grid, warps * 32, 0, st>>>(
-        idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-        argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft);
+    if (did_prewalk) {
+        accept_kernel<kTailResume><<<grid, warps * 32, 0, st>>>(
+            idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+            argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft,
+            sc.pre_state, sc.pre_len);
+    } else {
+        accept_kernel<kTailFullWalk><<<grid, warps * 32, 0, st>>>(
+            idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+            argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft,
+            nullptr, nullptr);
+    }
     SAM_CUDA(cudaGetLastError());
     prof_mark(2, st);
     prof_done();
@@ -348,7 +386,7 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     int rc = static_scratch(&keys);
     if (rc != SAM_OK) return rc;
     rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
-                           n_accepted, keys, static_cast<int64_t>(SAM_STATIC_MAX_ROWS) * 8 + 512);
+                           n_accepted, keys, INT64_MAX);   // the array is sized for SAM_STATIC_MAX_ROWS rows
     if (rc != SAM_OK || B == 0) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // whatever an earlier (possibly failed) call left behind, these rows start from zero
@@ -358,9 +396,9 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     if (rc != SAM_OK) return rc;
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    accept_kernel<false><<<grid, warps * 32, 0, st>>>(
+    accept_kernel<kTailVerifyOnly><<<grid, warps * 32, 0, st>>>(
         DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr);
+        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr, nullptr, nullptr);
     SAM_CUDA(cudaGetLastError());
     prof_mark(2, st);
     prof_done();

@@ -164,6 +164,41 @@ draft_kernel(DeviceSam sam, int B, int* __restrict__ state, int* __restrict__ ma
     }
 }
 
+// Walk-ahead along the draft.  While the logits of a step are still being reduced, spare warps
+// follow the automaton over each stream's DRAFT tokens and record the (state, matched_len)
+// reached after every prefix.  Whatever prefix the verification later accepts, the walk over it
+// is then already done and only the model's own token remains to be followed.
+struct PreWalk {
+    const int* state;        // [B] stream state at the start of the step
+    const int* matched_len;  // [B]
+    const int* drafts;       // [B, K]
+    const int* n_draft;      // [B]
+    int* pre_state;          // [B, K] state after drafts[b, 0..j]
+    int* pre_len;            // [B, K] matched_len after drafts[b, 0..j]
+    int B, K;
+    int enabled;
+};
+
+__device__ __forceinline__ void prewalk_stream(const DeviceSam& sam, const PreWalk& pw, int b, int lane) {
+    int s = pw.state[b];
+    int L = pw.matched_len[b];
+    sanitize_stream_state(sam, s, L);
+    const int nd = max(0, min(pw.n_draft[b], pw.K));
+    const int d = (lane < nd) ? pw.drafts[static_cast<long long>(b) * pw.K + lane] : -1;
+    if (nd == 0) return;
+    RecRegs r = (s == 0) ? root_rec() : load_rec(sam, s);
+    int my_s = 0, my_L = 0;
+    for (int j = 0; j < nd; ++j) {
+        const int c = __shfl_sync(kFull, d, j);
+        walk_token(sam, c, s, L, r, lane);
+        if (lane == j) { my_s = s; my_L = L; }
+    }
+    if (lane < nd) {
+        pw.pre_state[static_cast<long long>(b) * pw.K + lane] = my_s;
+        pw.pre_len[static_cast<long long>(b) * pw.K + lane] = my_L;
+    }
+}
+
 // ============================================================================================
 // Vocabulary argmax (Algorithm 3 "Validate with main LLM": the model's greedy choice per row).
 // Bandwidth-bound: every bf16 is read once. Ties go to the lowest index.
@@ -330,19 +365,32 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
 // the first mismatch, then follow the automaton over what was committed and draft again).
 // One warp per stream. Also decodes the packed argmax candidates and re-zeroes them.
 // ============================================================================================
-template <bool kWalk>
+enum : int { kTailVerifyOnly = 0, kTailFullWalk = 1, kTailResume = 2 };
+
+template <int kMode>
 __global__ void __launch_bounds__(128)
 accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long stride, int B, int K,
               const int* __restrict__ drafts, const int* __restrict__ n_draft,
               int* __restrict__ argmax_out, int* __restrict__ accepted, int* __restrict__ n_accepted,
               unsigned long long* __restrict__ keys,
               int* __restrict__ state, int* __restrict__ matched_len, int min_match,
-              int* __restrict__ next_drafts, int* __restrict__ next_n_draft) {
+              int* __restrict__ next_drafts, int* __restrict__ next_n_draft,
+              const int* __restrict__ pre_state, const int* __restrict__ pre_len) {
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= B) return;
     const int K1 = K + 1;
     const long long row0 = static_cast<long long>(b) * K1;
+    // independent loads first, so that they travel together
+    int ps = 0, pl = 0, s = 0, L = 0;
+    if (kMode != kTailVerifyOnly) {
+        s = state[b];
+        L = matched_len[b];
+    }
+    if (kMode == kTailResume && lane < K) {
+        ps = pre_state[static_cast<long long>(b) * K + lane];
+        pl = pre_len[static_cast<long long>(b) * K + lane];
+    }
 
     // rows j = lane and j = lane + 32 (K + 1 <= 33)
     int am[2] = {-1, -1};
@@ -374,14 +422,22 @@ accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long
     }
     if (lane == 0) n_accepted[b] = a + 1;
 
-    if (kWalk) {
-        int s = state[b];
-        int L = matched_len[b];
+    if (kMode != kTailVerifyOnly) {
         sanitize_stream_state(sam, s, L);
-        RecRegs r = (s == 0) ? root_rec() : load_rec(sam, s);
-        for (int t = 0; t < a; ++t) {
-            const int c = __shfl_sync(kFull, d, t);
-            walk_token(sam, c, s, L, r, lane);
+        RecRegs r;
+        if (kMode == kTailResume) {
+            // the walk over the accepted draft prefix was done ahead of time
+            if (a > 0) {
+                s = __shfl_sync(kFull, ps, a - 1);
+                L = __shfl_sync(kFull, pl, a - 1);
+            }
+            r = (s == 0) ? root_rec() : load_rec(sam, s);
+        } else {
+            r = (s == 0) ? root_rec() : load_rec(sam, s);
+            for (int t = 0; t < a; ++t) {
+                const int c = __shfl_sync(kFull, d, t);
+                walk_token(sam, c, s, L, r, lane);
+            }
         }
         walk_token(sam, bonus, s, L, r, lane);
         const int nn = emit_draft(sam, L, r, K, min_match, next_drafts + static_cast<long long>(b) * K, lane);
