@@ -35,8 +35,8 @@ METRIC = "sam_draft_verify_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
-# capture summarised under profiles/ (None until a capture exists for the current kernel)
-NCU_DRAM_BYTES_PER_ROW = None
+# capture summarised in profiles/launch_list_cfg2.md (config 2, argmax_bulk_kernel; traffic scales with rows)
+NCU_DRAM_BYTES_PER_ROW = 304415.2
 
 
 # ----------------------------------------------------------------------------- helpers
