@@ -123,17 +123,8 @@ class ClockSampler:
 
 def make_inputs_gpu(cfg, device):
     """Corpus (host) and the noise logits generated on the device (seeded torch generator)."""
-    import torch
     corpus = W.make_corpus(cfg)
-    g = torch.Generator(device=device)
-    g.manual_seed(1000 + cfg.seed)
-    R = cfg.rows
-    logits = torch.empty((R, cfg.vocab), dtype=torch.bfloat16, device=device)
-    blk = max(1, (1 << 26) // cfg.vocab)
-    for r0 in range(0, R, blk):
-        r1 = min(R, r0 + blk)
-        logits[r0:r1] = torch.randn((r1 - r0, cfg.vocab), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
-    rowmax = logits.max(dim=1).values.view(torch.int16).cpu().numpy().view(np.uint16)
+    logits, rowmax = W.make_noise_logits_device(cfg, device)
     return corpus, logits, rowmax
 
 
@@ -355,7 +346,7 @@ def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads)
 
 def cpu_baseline(cfg, corpus, scripts, logits_dev, rowmax, steps):
     import oracle
-    host_bits = logits_dev.view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+    host_bits = W.device_bits_to_host(logits_dev)
     threads = oracle.host_threads()
     tokens, secs, t_build = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, 1, steps, threads)
     return {"value": tokens / secs, "unit": UNIT, "cores": threads, "kind": "oracle",

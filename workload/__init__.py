@@ -18,3 +18,4 @@ from .agent_memory import (  # noqa: F401
     zipf_cdf,
 )
 from .closed_loop import HostLogits, run_closed_loop, trace_stats  # noqa: F401,E402
+from .device_noise import device_bits_to_host, make_noise_logits_device  # noqa: F401,E402
