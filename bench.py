@@ -147,11 +147,12 @@ def run_ours(args):
         build()
     if world > 1:
         dist.barrier()
+    S.sam_set_argmax_variant(args.variant)
 
     base = W.CONFIGS[args.config]
     # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
     # read-only automaton is replicated; no data-path collective
-    cfg = base.scaled(steps=args.warmup + args.steps + args.e2e_steps + 1)
+    cfg = base.scaled(steps=args.warmup + args.steps + args.split_steps + args.e2e_steps + 1)
     stream_cfg = cfg.scaled(seed=cfg.seed + 7919 * rank) if rank > 0 else cfg
 
     t0 = time.time()
@@ -207,7 +208,7 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    S.sam_profile_enable(args.steps)
+    launches0 = S.sam_launch_count()
     wall0 = time.time()
     for i in range(args.steps):
         one_step(args.warmup + i, timed_slot=i)
@@ -215,13 +216,41 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     wall = time.time() - wall0
+    launches = S.sam_launch_count() - launches0
     clocks = sampler.stop(wall0, wall0 + wall) if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    prof = [S.sam_profile_read(i) for i in range(S.sam_profile_count())]
-    S.sam_profile_enable(0)
     total_ms = float(sum(step_ms))
-    argmax_ms = statistics.mean(p[0] for p in prof)
-    accept_ms = statistics.mean(p[1] for p in prof)
+    launches_per_step = launches / args.steps
+
+    # ---- per-kernel split, outside the timed region: the same loop continues with the accept step in a kernel
+    # of its own, so that the library's events separate the vocabulary argmax from accept + walk + draft
+    split = None
+    if args.split_steps > 0:
+        S.sam_set_argmax_variant(3 if args.variant == 0 else args.variant)
+        S.sam_profile_enable(args.split_steps)
+        n_before = len(stats_trace)
+        for i in range(args.split_steps):
+            t = args.warmup + args.steps + i
+            ow = feeder.overwrites(t, drafts, n_draft)
+            saved = be.poke(ow["row"], ow["col"], ow["bits"], np.arange(ow["row"].shape[0]))
+            in_nd = n_draft
+            torch.cuda._sleep(args.presleep_cycles)
+            be.launch_step()
+            torch.cuda.synchronize()
+            n_acc = be.n_accepted.cpu().numpy()
+            drafts, n_draft = be.drafts.cpu().numpy(), be.n_draft.cpu().numpy()
+            be.unpoke(ow["row"], ow["col"], saved)
+            feeder.advance(n_acc)
+            stats_trace.append(dict(n_accepted=n_acc, in_n_draft=in_nd))
+        sp = [S.sam_profile_read(i) for i in range(S.sam_profile_count())]
+        S.sam_profile_enable(0)
+        S.sam_set_argmax_variant(args.variant)
+        split_trace = stats_trace[n_before:]
+        del stats_trace[n_before:]
+        split = {"steps": args.split_steps, "argmax_ms": statistics.mean(p[0] for p in sp),
+                 "accept_walk_draft_ms": statistics.mean(p[1] for p in sp),
+                 "committed": int(sum(int(o["n_accepted"].sum()) for o in split_trace)),
+                 "drafted": int(sum(int(o["in_n_draft"].sum()) for o in split_trace))}
 
     # ---- end to end through the host-buffer entry point: logits and bookkeeping start in pinned host memory
     e2e = None
@@ -277,7 +306,21 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
     R = cfg.rows
     alg_bytes = R * (2 * cfg.vocab + 4)
-    achieved = alg_bytes / (argmax_ms * 1e-3) / 1e9
+    # dominant kernel: with one launch per step the step's event bracket IS that kernel's duration (vocabulary
+    # argmax with the accept / walk / draft tail inside); with two launches per step the argmax kernel's own
+    # time comes from the split measurement
+    if launches_per_step == 1:
+        kernel_ms, kernel_name = total_ms / args.steps, "argmax_bulk_kernel (argmax + fused accept/walk/draft tail)"
+    else:
+        kernel_ms, kernel_name = (split["argmax_ms"] if split else total_ms / args.steps), "argmax kernel alone"
+    achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
+    walk = None
+    if split is not None:
+        walk_s = split["accept_walk_draft_ms"] * split["steps"] / 1e3
+        walk = {"draft_tokens_per_s": split["drafted"] / walk_s, "committed_tokens_per_s_kernel_only": split["committed"] / walk_s,
+                "argmax_only_GBps": alg_bytes / (split["argmax_ms"] * 1e-3) / 1e9,
+                "note": f"{split['steps']} further steps of the same loop after the timed region, accept + walk + draft "
+                        "in a kernel of its own (library events around it)", **split}
     st = W.trace_stats(cfg, stats_trace)
     out = {
         "metric": METRIC, "value": all_tokens / (max_ms / 1e3), "unit": UNIT,
@@ -294,14 +337,13 @@ def run_ours(args):
                              "event keeps the queue full so host launch latency is not timed"},
         "steps_per_s": args.steps / (max_ms / 1e3),
         "stream_steps_per_s": world * cfg.B * args.steps / (max_ms / 1e3),
-        "gpu_launches": 2 * args.steps,
-        "kernels_ms": {"argmax": argmax_ms, "accept_walk_draft": accept_ms},
-        "roofline": {"kernel": "argmax", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "gpu_launches": launches,
+        "launches_per_step": launches_per_step, "variant": args.variant,
+        "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
                      "traffic": (NCU_DRAM_BYTES_PER_ROW * R) if NCU_DRAM_BYTES_PER_ROW else None,
                      "algorithmic_bytes": alg_bytes},
-        "walk": {"draft_tokens_per_s": st["mean_n_draft"] * cfg.B * args.steps / (accept_ms * args.steps / 1e3),
-                 "committed_tokens_per_s_kernel_only": tokens / (accept_ms * args.steps / 1e3)},
+        "walk": walk,
         "ote": st["ote"], "shr": st["shr"], "mean_n_draft": st["mean_n_draft"],
         "e2e": e2e, "clocks": clocks,
         "setup_s": {"inputs": t_inputs, "sam_build": t_build, "sam_upload": t_upload,
@@ -396,6 +438,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--presleep-cycles", type=int, default=300000,
                     help="length of the spin kernel enqueued before each timed step (outside the events)")
+    ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 3],
+                    help="kernel selection of the library (0 = default: one fused kernel per step; "
+                         "3 = argmax and accept as two kernels; 1 = direct-load argmax + accept)")
+    ap.add_argument("--split-steps", type=int, default=20,
+                    help="steps run after the timed region with two kernels per step, to report each kernel's time")
     ap.add_argument("--cpu-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     args = ap.parse_args()

@@ -87,7 +87,8 @@ void sam_free(sam_index* idx);
 /* ---------------------------------------------------------------- verification scratch */
 
 /* Bytes of device scratch sam_verify / sam_step need for B streams and draft length K
- * (one 64-bit partial result per logits row).  Returns a negative SAM_ERR_* on bad sizes. */
+ * (one 64-bit partial result per logits row, the walk-ahead states of every draft position, one
+ * completion counter per stream and a status word).  Returns a negative SAM_ERR_* on bad sizes. */
 int64_t sam_workspace_bytes(int32_t B, int32_t K);
 
 /* Zero-fills the scratch (device, 8-byte aligned) on the stream.  Required once before the
@@ -97,10 +98,11 @@ int64_t sam_workspace_bytes(int32_t B, int32_t K);
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
 
 /* Reads the status word the verification kernels keep at the end of the scratch: 0 = fine,
- * 1 = a kernel gave up on one of its internal (bounded) waits and the outputs of that call are
- * not valid - re-initialise the scratch and retry.  Copies one int to the host and synchronises
- * the stream: a diagnostic, not a hot-path call.  B and K locate the word (same values as in
- * the calls that used the scratch). */
+ * 1 = a kernel gave up on one of its internal (bounded) waits, 2 = a kernel was handed more
+ * finished streams than its internal queue holds (the host sizes the launch so that this does not
+ * happen).  After a non-zero status the outputs of that call are not valid - re-initialise the
+ * scratch and retry.  Copies one int to the host and synchronises the stream: a diagnostic, not a
+ * hot-path call.  B and K locate the word (same values as in the calls that used the scratch). */
 int sam_workspace_status(const void* workspace, int32_t B, int32_t K, int32_t* status_out, void* cuda_stream);
 
 /* ---------------------------------------------------------------- hot path (device, async) */
@@ -211,12 +213,18 @@ int sam_step_host(const sam_index* idx,
  * milliseconds; the stream must have been synchronised by the caller first.
  * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
 int sam_profile_enable(int32_t max_calls);
-/* Selects the argmax kernel for later calls (process-wide; for measurements and tests):
- * 0 = by alignment (default: bulk-copy pipeline when the logits base and row stride are 16-byte
- * aligned, direct loads otherwise), 1 = always direct loads, 2 = same as 0. */
+/* Selects the kernels of sam_verify / sam_step for later calls (process-wide; for measurements
+ * and tests): 0 = by alignment (default: when the logits base and row stride are 16-byte aligned,
+ * one bulk-copy pipelined kernel that also runs the accept step of every stream as soon as its
+ * rows are complete; direct loads plus a separate accept kernel otherwise), 1 = always direct
+ * loads, 2 = same as 0, 3 = as 0 but with the accept step in a kernel of its own. */
 int sam_set_argmax_variant(int32_t variant);
 int32_t sam_profile_count(void);
 int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms);
+
+/* Number of kernels this library has enqueued in this process so far (all entry points, all
+ * threads); a measurement aid with no counterpart in the paper. */
+int64_t sam_launch_count(void);
 
 /* Static description of a status code. */
 const char* sam_strerror(int status);

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     sam_export,
     sam_free,
     sam_last_cuda_error,
+    sam_launch_count,
     sam_profile_count,
     sam_profile_enable,
     sam_profile_read,

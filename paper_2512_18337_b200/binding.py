@@ -48,6 +48,7 @@ _SIGNATURES = {
     "sam_profile_read": (C.c_int, [_i32, C.POINTER(C.c_float), C.POINTER(C.c_float)]),
     "sam_strerror": (C.c_char_p, [C.c_int]),
     "sam_last_cuda_error": (C.c_int, []),
+    "sam_launch_count": (_i64, []),
 }
 
 
@@ -261,6 +262,10 @@ def sam_strerror(status: int) -> str:
 
 def sam_last_cuda_error() -> int:
     return int(_load().sam_last_cuda_error())
+
+
+def sam_launch_count() -> int:
+    return int(_load().sam_launch_count())
 
 
 # ------------------------------------------------------------------ convenience holder

@@ -3,6 +3,7 @@
 
 #include <cstdint>
 #include <cstdlib>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -18,6 +19,7 @@ using namespace samb200;
 namespace {
 
 thread_local int g_last_cuda = 0;
+std::atomic<long long> g_launches{0};   // kernels this library has enqueued (diagnostic)
 
 inline int cuda_fail(cudaError_t e) {
     g_last_cuda = static_cast<int>(e);
@@ -76,7 +78,7 @@ int check_verify_args(const void* logits, int64_t stride, int32_t B, int32_t K, 
     return SAM_OK;
 }
 
-int g_argmax_variant = 0;   // 0 = choose by alignment, 1 = direct loads, 2 = bulk-copy pipeline (if alignment allows)
+int g_argmax_variant = 0;   // 0/2 = choose by alignment, 1 = direct loads always, 3 = as 0 but the accept step in its own kernel
 
 inline int* status_word(unsigned long long* keys, int64_t R) {
     return reinterpret_cast<int*>(reinterpret_cast<char*>(keys) + ((R * 8 + 255) / 256) * 256);
@@ -84,12 +86,13 @@ inline int* status_word(unsigned long long* keys, int64_t R) {
 
 // Partial results land in keys[R]; `status` receives a non-zero code if a kernel gives up on an
 // internal wait.
-// Layout of the verification scratch: keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K]
+// Layout of the verification scratch: keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B]
 struct Scratch {
     unsigned long long* keys;
     int* status;
     int* pre_state;
     int* pre_len;
+    int* done;
     int64_t bytes;
 };
 Scratch scratch_layout(void* base, int32_t B, int32_t K) {
@@ -102,21 +105,27 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K) {
     s.status = reinterpret_cast<int*>(p + o);               o += 256;
     s.pre_state = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * K * 4);
     s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * K * 4);
+    s.done = reinterpret_cast<int*>(p + o);                 o = up(o + static_cast<int64_t>(B) * 4);
     s.bytes = o;
     return s;
 }
 
-// Enqueues the argmax over R rows (and, when pw.enabled and the bulk kernel runs, the walk-ahead
-// along the drafts).  *did_prewalk tells the caller whether pre_state / pre_len will be filled.
+// Enqueues the argmax over R rows.  With the bulk-copy kernel two more things can ride along:
+// the walk-ahead over the drafts (pw) and the accept step of every stream (tail; needs `done`).
+// *did_prewalk / *did_tail tell the caller what the launch will have done; whatever it did not do
+// is left to a separate accept kernel.
 int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
                   int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
-                  bool* did_prewalk = nullptr) {
+                  bool* did_prewalk = nullptr, const AcceptArgs* tail = nullptr, int tail_mode = 0,
+                  int* done = nullptr, bool* did_tail = nullptr) {
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != SAM_OK) return rc;
     const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0;
     const bool bulk = rows_aligned && g_argmax_variant != 1;
+    if (did_prewalk) *did_prewalk = false;
+    if (did_tail) *did_tail = false;
     if (bulk) {
         static thread_local int attr_dev = -1;
         int dev = 0;
@@ -133,10 +142,26 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         int64_t grid = di.sms;
         if (grid > total) grid = total;
         if (grid < 1) grid = 1;
+        const bool prewalk = pw != nullptr && pw->enabled != 0;
+        FusedTail ft{};
+        if (tail != nullptr && done != nullptr && g_argmax_variant != 3) {
+            // a CTA can be handed at most the streams that overlap its contiguous range of rows
+            const int64_t rows_per_cta = (total + grid - 1) / grid / tiles_per_row + 2;
+            const int64_t streams_per_cta = rows_per_cta / (tail->K + 1) + 2;
+            const int64_t expected = static_cast<int64_t>(tiles_per_row) * (tail->K + 1) + (prewalk ? 1 : 0);
+            if (streams_per_cta <= kQueueCap && expected < (int64_t(1) << 30)) {
+                ft.args = *tail;
+                ft.done = done;
+                ft.expected = static_cast<int>(expected);
+                ft.mode = tail_mode + 1;
+            }
+        }
         argmax_bulk_kernel<<<static_cast<unsigned>(grid), kBulkThreads, kBulkSmemBytes, st>>>(
             static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status,
-            sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{});
-        if (did_prewalk) *did_prewalk = (pw != nullptr && pw->enabled != 0);
+            sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{}, ft);
+        ++g_launches;
+        if (did_prewalk) *did_prewalk = prewalk;
+        if (did_tail) *did_tail = ft.mode != 0;
     } else {
         const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
         const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
@@ -146,9 +171,20 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid < 1) grid = 1;
         argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
             static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys);
+        ++g_launches;
     }
     SAM_CUDA(cudaGetLastError());
     prof_mark(1, st);
+    return SAM_OK;
+}
+
+template <int kMode>
+int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st) {
+    const int warps = 4;
+    const unsigned grid = static_cast<unsigned>((a.B + warps - 1) / warps);
+    accept_kernel<kMode><<<grid, warps * 32, 0, st>>>(sam, a);
+    ++g_launches;
+    SAM_CUDA(cudaGetLastError());
     return SAM_OK;
 }
 
@@ -255,6 +291,7 @@ int sam_draft(const sam_index* idx, int32_t B, int32_t* state, int32_t* matched_
     const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
     draft_kernel<<<grid, warps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         idx->dev, B, state, matched_len, new_tokens, ld, n_new, K, min_match, drafts, n_draft);
+    ++g_launches;
     SAM_CUDA(cudaGetLastError());
     return SAM_OK;
 }
@@ -267,16 +304,19 @@ int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int
                                n_accepted, workspace, workspace_bytes);
     if (rc != SAM_OK || B == 0) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    unsigned long long* keys = static_cast<unsigned long long*>(workspace);
     const int64_t R = static_cast<int64_t>(B) * (K + 1);
-    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, status_word(keys, R), st);
+    const Scratch sc = scratch_layout(workspace, B, K);
+    const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                        argmax_out, accepted, n_accepted, sc.keys, nullptr, nullptr, 1, nullptr, nullptr,
+                        nullptr, nullptr};
+    bool did_tail = false;
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, nullptr, nullptr, nullptr,
+                       &aa, kTailVerifyOnly, sc.done, &did_tail);
     if (rc != SAM_OK) return rc;
-    const int warps = 4;
-    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    accept_kernel<kTailVerifyOnly><<<grid, warps * 32, 0, st>>>(
-        DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr, nullptr, nullptr);
-    SAM_CUDA(cudaGetLastError());
+    if (!did_tail) {
+        rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
+        if (rc != SAM_OK) return rc;
+    }
     prof_mark(2, st);
     prof_done();
     return SAM_OK;
@@ -297,27 +337,20 @@ int sam_step(const sam_index* idx,
     if (B == 0) return SAM_OK;
     if (!state || !matched_len || !next_drafts || !next_n_draft) return SAM_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    unsigned long long* keys = static_cast<unsigned long long*>(workspace);
     const int64_t R = static_cast<int64_t>(B) * (K + 1);
     const Scratch sc = scratch_layout(workspace, B, K);
     PreWalk pw{state, matched_len, drafts, n_draft, sc.pre_state, sc.pre_len, B, K, 1};
-    bool did_prewalk = false;
-    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, keys, sc.status, st, &idx->dev, &pw, &did_prewalk);
+    AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                  argmax_out, accepted, n_accepted, sc.keys, state, matched_len, min_match, next_drafts,
+                  next_n_draft, sc.pre_state, sc.pre_len};
+    bool did_prewalk = false, did_tail = false;
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, &idx->dev, &pw, &did_prewalk,
+                       &aa, kTailResume, sc.done, &did_tail);
     if (rc != SAM_OK) return rc;
-    const int warps = 4;
-    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    if (did_prewalk) {
-        accept_kernel<kTailResume><<<grid, warps * 32, 0, st>>>(
-            idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-            argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft,
-            sc.pre_state, sc.pre_len);
-    } else {
-        accept_kernel<kTailFullWalk><<<grid, warps * 32, 0, st>>>(
-            idx->dev, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-            argmax_out, accepted, n_accepted, keys, state, matched_len, min_match, next_drafts, next_n_draft,
-            nullptr, nullptr);
+    if (!did_tail) {
+        rc = did_prewalk ? launch_accept<kTailResume>(idx->dev, aa, st) : launch_accept<kTailFullWalk>(idx->dev, aa, st);
+        if (rc != SAM_OK) return rc;
     }
-    SAM_CUDA(cudaGetLastError());
     prof_mark(2, st);
     prof_done();
     return SAM_OK;
@@ -394,12 +427,11 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     rc = launch_argmax(logits_bf16, row_stride_elems, rows, V, keys,
                        reinterpret_cast<int*>(keys + SAM_STATIC_MAX_ROWS), st);
     if (rc != SAM_OK) return rc;
-    const int warps = 4;
-    const unsigned grid = static_cast<unsigned>((B + warps - 1) / warps);
-    accept_kernel<kTailVerifyOnly><<<grid, warps * 32, 0, st>>>(
-        DeviceSam{}, static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr, nullptr, nullptr);
-    SAM_CUDA(cudaGetLastError());
+    const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                        argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr,
+                        nullptr, nullptr};
+    rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
+    if (rc != SAM_OK) return rc;
     prof_mark(2, st);
     prof_done();
     return SAM_OK;
@@ -493,7 +525,7 @@ int sam_workspace_status(const void* workspace, int32_t B, int32_t K, int32_t* s
 }
 
 int sam_set_argmax_variant(int32_t variant) {
-    if (variant < 0 || variant > 2) return SAM_ERR_INVALID_ARG;
+    if (variant < 0 || variant > 3) return SAM_ERR_INVALID_ARG;
     g_argmax_variant = variant;
     return SAM_OK;
 }
@@ -512,5 +544,7 @@ const char* sam_strerror(int status) {
 }
 
 int sam_last_cuda_error(void) { return g_last_cuda; }
+
+int64_t sam_launch_count(void) { return g_launches.load(); }
 
 }  // extern "C"

@@ -217,6 +217,12 @@ __device__ __forceinline__ unsigned long long pack_candidate(float x, unsigned i
     return (static_cast<unsigned long long>(ordered_key(x)) << 32) | (0xFFFFFFFFu - idx);
 }
 
+// A row whose element 0 is NaN keeps index 0 (nothing ever compares greater than NaN): this
+// candidate beats every real one (value keys stop at 0xFF80) and decodes to index 0.
+constexpr unsigned long long kCandidateFirstIsNaN = 0x0000FFFFFFFFFFFFull;
+
+__device__ __forceinline__ bool bf16_bits_nan(unsigned b) { return (b & 0x7FFFu) > 0x7F80u; }
+
 __device__ __forceinline__ float bf16lo(unsigned u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi(unsigned u) { return __uint_as_float(u & 0xFFFF0000u); }
 
@@ -321,10 +327,11 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
     RowView rv{};
     float best = __int_as_float(0xff800000);   // -inf: only strictly greater values become candidates
     int bestq = -1;
+    bool first_nan = false;                    // this thread saw a NaN in element 0 of the current row
 
     auto flush = [&]() {
         if (cur_row < 0) return;
-        unsigned long long k = resolve_candidate(rv, V, best, bestq);
+        unsigned long long k = first_nan ? kCandidateFirstIsNaN : resolve_candidate(rv, V, best, bestq);
         k = warp_max_u64(k);
         if (lane == 0 && k != 0ull) atomicMax(keys + cur_row, k);
     };
@@ -338,6 +345,7 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
             rv = row_view(logits, stride, row, V);
             best = __int_as_float(0xff800000);
             bestq = -1;
+            first_nan = false;
         }
         const int q0 = tile * kTileVec + threadIdx.x;
         uint4 v[kVecPerThread];
@@ -351,6 +359,11 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
         for (int i = 0; i < kVecPerThread; ++i) {
             const int q = q0 + i * kArgmaxThreads;
             if (q < rv.nvec) {
+                if (q == 0) {
+                    const int h = rv.off >> 1;
+                    const unsigned pair = (h == 0) ? v[i].x : (h == 1) ? v[i].y : (h == 2) ? v[i].z : v[i].w;
+                    first_nan = bf16_bits_nan((rv.off & 1) ? (pair >> 16) : (pair & 0xFFFFu));
+                }
                 if (q == 0 || q == rv.nvec - 1) mask_vector(v[i], q, rv.off, V);
                 const float m = vec_max(v[i]);
                 if (m > best) { best = m; bestq = q; }
@@ -367,29 +380,49 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
 // ============================================================================================
 enum : int { kTailVerifyOnly = 0, kTailFullWalk = 1, kTailResume = 2 };
 
+// Everything the accept step of one stream reads and writes (device pointers of the caller).
+struct AcceptArgs {
+    const __nv_bfloat16* logits;
+    long long stride;
+    int B, K;
+    const int* drafts;        // [B, K]
+    const int* n_draft;       // [B]
+    int* argmax_out;          // [B, K+1]
+    int* accepted;            // [B, K+1]
+    int* n_accepted;          // [B]
+    unsigned long long* keys; // [B*(K+1)] packed argmax candidates, re-zeroed here
+    int* state;               // [B] (unused in kTailVerifyOnly)
+    int* matched_len;         // [B]
+    int min_match;
+    int* next_drafts;         // [B, K]
+    int* next_n_draft;        // [B]
+    const int* pre_state;     // [B, K] walk-ahead results (kTailResume)
+    const int* pre_len;       // [B, K]
+};
+
+// One warp, one stream.  The packed candidates and the walk-ahead results may have been produced
+// by other SMs moments ago, so they are read past L1 (ld.cg).
 template <int kMode>
-__global__ void __launch_bounds__(128)
-accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long stride, int B, int K,
-              const int* __restrict__ drafts, const int* __restrict__ n_draft,
-              int* __restrict__ argmax_out, int* __restrict__ accepted, int* __restrict__ n_accepted,
-              unsigned long long* __restrict__ keys,
-              int* __restrict__ state, int* __restrict__ matched_len, int min_match,
-              int* __restrict__ next_drafts, int* __restrict__ next_n_draft,
-              const int* __restrict__ pre_state, const int* __restrict__ pre_len) {
-    const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (b >= B) return;
+__device__ __forceinline__ void accept_stream(const DeviceSam& sam, const AcceptArgs& p, int b, int lane) {
+    const int K = p.K;
     const int K1 = K + 1;
     const long long row0 = static_cast<long long>(b) * K1;
     // independent loads first, so that they travel together
     int ps = 0, pl = 0, s = 0, L = 0;
+    RecRegs r = root_rec();
     if (kMode != kTailVerifyOnly) {
-        s = state[b];
-        L = matched_len[b];
+        s = p.state[b];
+        L = p.matched_len[b];
+        sanitize_stream_state(sam, s, L);
+        if (s != 0) r = load_rec(sam, s);
     }
-    if (kMode == kTailResume && lane < K) {
-        ps = pre_state[static_cast<long long>(b) * K + lane];
-        pl = pre_len[static_cast<long long>(b) * K + lane];
+    const int nd = max(0, min(p.n_draft[b], K));
+    RecRegs rj = root_rec();     // kTailResume: lane j fetches the record of the state reached after j + 1 drafts
+    if (kMode == kTailResume && lane < nd) {
+        ps = __ldcg(p.pre_state + static_cast<long long>(b) * K + lane);
+        pl = __ldcg(p.pre_len + static_cast<long long>(b) * K + lane);
+        // every possible resume point is fetched now, while the row results are still on their way
+        if (ps > 0 && ps < sam.n_states) rj = load_rec(sam, ps);
     }
 
     // rows j = lane and j = lane + 32 (K + 1 <= 33)
@@ -398,18 +431,16 @@ accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long
     for (int h = 0; h < 2; ++h) {
         const int j = lane + 32 * h;
         if (j < K1) {
-            const unsigned long long k = keys[row0 + j];
-            keys[row0 + j] = 0ull;
-            int idx = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
-            const unsigned short x0 = __ldg(reinterpret_cast<const unsigned short*>(logits + (row0 + j) * stride));
-            if ((x0 & 0x7FFFu) > 0x7F80u) idx = 0;     // element 0 is NaN: nothing ever compares greater
+            const unsigned long long k = __ldcg(p.keys + row0 + j);
+            p.keys[row0 + j] = 0ull;
+            // no candidate at all (nothing in the row is greater than -inf): index 0, as a scan from element 0 gives
+            const int idx = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
             am[h] = idx;
-            argmax_out[row0 + j] = idx;
+            p.argmax_out[row0 + j] = idx;
         }
     }
 
-    const int nd = max(0, min(n_draft[b], K));
-    const int d = (lane < K) ? drafts[static_cast<long long>(b) * K + lane] : -1;
+    const int d = (lane < K) ? p.drafts[static_cast<long long>(b) * K + lane] : -1;
     const unsigned mism = __ballot_sync(kFull, lane < nd && d != am[0]);
     const int a = mism ? (__ffs(mism) - 1) : nd;        // accepted draft tokens
     const int bonus_lo = __shfl_sync(kFull, am[0], a & 31);
@@ -418,35 +449,45 @@ accept_kernel(DeviceSam sam, const __nv_bfloat16* __restrict__ logits, long long
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int j = lane + 32 * h;
-        if (j < K1) accepted[row0 + j] = (j < a) ? d : ((j == a) ? bonus : -1);
+        if (j < K1) p.accepted[row0 + j] = (j < a) ? d : ((j == a) ? bonus : -1);
     }
-    if (lane == 0) n_accepted[b] = a + 1;
+    if (lane == 0) p.n_accepted[b] = a + 1;
 
     if (kMode != kTailVerifyOnly) {
-        sanitize_stream_state(sam, s, L);
-        RecRegs r;
         if (kMode == kTailResume) {
             // the walk over the accepted draft prefix was done ahead of time
             if (a > 0) {
-                s = __shfl_sync(kFull, ps, a - 1);
-                L = __shfl_sync(kFull, pl, a - 1);
+                const int src = a - 1;
+                s = __shfl_sync(kFull, ps, src);
+                L = __shfl_sync(kFull, pl, src);
+                r.a.x = __shfl_sync(kFull, rj.a.x, src); r.a.y = __shfl_sync(kFull, rj.a.y, src);
+                r.a.z = __shfl_sync(kFull, rj.a.z, src); r.a.w = __shfl_sync(kFull, rj.a.w, src);
+                r.b.x = __shfl_sync(kFull, rj.b.x, src); r.b.y = __shfl_sync(kFull, rj.b.y, src);
+                r.b.z = __shfl_sync(kFull, rj.b.z, src); r.b.w = __shfl_sync(kFull, rj.b.w, src);
             }
-            r = (s == 0) ? root_rec() : load_rec(sam, s);
         } else {
-            r = (s == 0) ? root_rec() : load_rec(sam, s);
             for (int t = 0; t < a; ++t) {
                 const int c = __shfl_sync(kFull, d, t);
                 walk_token(sam, c, s, L, r, lane);
             }
         }
         walk_token(sam, bonus, s, L, r, lane);
-        const int nn = emit_draft(sam, L, r, K, min_match, next_drafts + static_cast<long long>(b) * K, lane);
+        const int nn = emit_draft(sam, L, r, K, p.min_match, p.next_drafts + static_cast<long long>(b) * K, lane);
         if (lane == 0) {
-            state[b] = s;
-            matched_len[b] = L;
-            next_n_draft[b] = nn;
+            p.state[b] = s;
+            p.matched_len[b] = L;
+            p.next_n_draft[b] = nn;
         }
     }
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(128)
+accept_kernel(DeviceSam sam, AcceptArgs p) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= p.B) return;
+    accept_stream<kMode>(sam, p, b, lane);
 }
 
 }  // namespace samb200

@@ -53,7 +53,9 @@ def _check_verify(bits, V, B, K, rng):
         keep = rng.random(nd) < 0.8
         drafts[b, :nd] = np.where(keep, am_o[b, :nd], rng.integers(0, V, size=nd))
     acc_o, nacc_o = oracle.accept_batch(drafts, n_draft, am_o)
-    for variant in (0, 1):     # 0: bulk-copy pipeline when rows are 16-byte aligned; 1: direct loads always
+    # 0: bulk-copy pipeline with the accept step fused in (when rows are 16-byte aligned);
+    # 1: direct loads always; 3: bulk-copy pipeline, accept step in its own kernel
+    for variant in (0, 1, 3):
         am, acc, nacc = _verify_gpu(bits, V, B, K, drafts, n_draft, variant=variant)
         assert (am == am_o).all(), variant
         assert (nacc == nacc_o).all() and (acc == acc_o).all(), variant
@@ -250,6 +252,26 @@ def test_closed_loop_tiny():
 def test_closed_loop_cfg1_full():
     """Config 1 at its full size: 1M-token corpus, B=64, K=8, V=151,936, all 64 steps."""
     cfg = W.CONFIGS[1]
+    tr_o, tr_g = _closed_loop_pair(cfg)
+    _assert_traces_equal(tr_o, tr_g)
+
+
+@pytest.mark.parametrize("variant", [1, 3])
+def test_closed_loop_other_kernel_variants(variant):
+    """The fused step with direct loads (full walk in the accept kernel) and with the bulk-copy argmax
+    followed by a separate accept kernel (walk-ahead resumed) gives the same trace as the oracle."""
+    cfg = W.CONFIGS[2].scaled(sessions=64, B=300, steps=6)
+    S.sam_set_argmax_variant(variant)
+    try:
+        tr_o, tr_g = _closed_loop_pair(cfg)
+    finally:
+        S.sam_set_argmax_variant(0)
+    _assert_traces_equal(tr_o, tr_g)
+
+
+def test_closed_loop_many_streams_per_cta():
+    """Short rows and many streams: every CTA finishes dozens of streams inside the argmax kernel."""
+    cfg = W.CONFIGS[0].scaled(B=3000, K=2, steps=5, vocab=1000)
     tr_o, tr_g = _closed_loop_pair(cfg)
     _assert_traces_equal(tr_o, tr_g)
 
