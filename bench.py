@@ -226,7 +226,7 @@ def run_ours(args):
     # of its own, so that the library's events separate the vocabulary argmax from accept + walk + draft
     split = None
     if args.split_steps > 0:
-        S.sam_set_argmax_variant(3 if args.variant == 0 else args.variant)
+        S.sam_set_argmax_variant(0 if args.variant == 2 else args.variant)
         S.sam_profile_enable(args.split_steps)
         n_before = len(stats_trace)
         for i in range(args.split_steps):
@@ -438,10 +438,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--presleep-cycles", type=int, default=300000,
                     help="length of the spin kernel enqueued before each timed step (outside the events)")
-    ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 3],
-                    help="kernel selection of the library (0 = default: one fused kernel per step; "
-                         "3 = argmax and accept as two kernels; 1 = direct-load argmax + accept)")
-    ap.add_argument("--split-steps", type=int, default=20,
+    ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 2],
+                    help="kernel selection of the library (0 = default: bulk-copy argmax kernel + accept kernel; "
+                         "1 = direct-load argmax + accept; 2 = one kernel per step with the accept step inside)")
+    ap.add_argument("--split-steps", type=int, default=50,
                     help="steps run after the timed region with two kernels per step, to report each kernel's time")
     ap.add_argument("--cpu-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

@@ -214,10 +214,11 @@ int sam_step_host(const sam_index* idx,
  * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
 int sam_profile_enable(int32_t max_calls);
 /* Selects the kernels of sam_verify / sam_step for later calls (process-wide; for measurements
- * and tests): 0 = by alignment (default: when the logits base and row stride are 16-byte aligned,
- * one bulk-copy pipelined kernel that also runs the accept step of every stream as soon as its
- * rows are complete; direct loads plus a separate accept kernel otherwise), 1 = always direct
- * loads, 2 = same as 0, 3 = as 0 but with the accept step in a kernel of its own. */
+ * and tests): 0 = by alignment (default: a bulk-copy pipelined argmax kernel when the logits base
+ * and row stride are 16-byte aligned, a direct-load kernel otherwise, each followed by the accept
+ * kernel), 1 = always direct loads, 2 = as 0, but the bulk-copy kernel also runs the accept step of
+ * every stream as soon as its rows are complete (one launch per call; measured slightly slower than
+ * two launches on B200), 3 = same as 0. */
 int sam_set_argmax_variant(int32_t variant);
 int32_t sam_profile_count(void);
 int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms);

@@ -78,7 +78,7 @@ int check_verify_args(const void* logits, int64_t stride, int32_t B, int32_t K, 
     return SAM_OK;
 }
 
-int g_argmax_variant = 0;   // 0/2 = choose by alignment, 1 = direct loads always, 3 = as 0 but the accept step in its own kernel
+int g_argmax_variant = 0;   // 0/3 = choose by alignment, 1 = direct loads always, 2 = as 0 with the accept step inside the argmax kernel
 
 inline int* status_word(unsigned long long* keys, int64_t R) {
     return reinterpret_cast<int*>(reinterpret_cast<char*>(keys) + ((R * 8 + 255) / 256) * 256);
@@ -144,7 +144,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid < 1) grid = 1;
         const bool prewalk = pw != nullptr && pw->enabled != 0;
         FusedTail ft{};
-        if (tail != nullptr && done != nullptr && g_argmax_variant != 3) {
+        if (tail != nullptr && done != nullptr && g_argmax_variant == 2) {
             // a CTA can be handed at most the streams that overlap its contiguous range of rows
             const int64_t rows_per_cta = (total + grid - 1) / grid / tiles_per_row + 2;
             const int64_t streams_per_cta = rows_per_cta / (tail->K + 1) + 2;
