@@ -36,7 +36,9 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
 # capture summarised in profiles/launch_list_cfg2.md (config 2, argmax_bulk_kernel; traffic scales with rows)
-NCU_DRAM_BYTES_PER_ROW = 304415.2
+NCU_DRAM_BYTES_PER_ROW = 304306.2
+# dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
+NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 112.7
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -319,6 +321,10 @@ def run_ours(args):
         walk_s = split["accept_walk_draft_ms"] * split["steps"] / 1e3
         walk = {"draft_tokens_per_s": split["drafted"] / walk_s, "committed_tokens_per_s_kernel_only": split["committed"] / walk_s,
                 "argmax_only_GBps": alg_bytes / (split["argmax_ms"] * 1e-3) / 1e9,
+                "bound": "latency (dependent random accesses)",
+                "dram_sector_GBps": NCU_ACCEPT_DRAM_SECTORS_PER_STREAM * cfg.B * 32 / (split["accept_walk_draft_ms"] * 1e-3) / 1e9,
+                "dram_sector_frac_of_peak": NCU_ACCEPT_DRAM_SECTORS_PER_STREAM * cfg.B * 32
+                                            / (split["accept_walk_draft_ms"] * 1e-3) / 1e9 / peak,
                 "note": f"{split['steps']} further steps of the same loop after the timed region, accept + walk + draft "
                         "in a kernel of its own (library events around it)", **split}
     st = W.trace_stats(cfg, stats_trace)
