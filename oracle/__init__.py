@@ -41,6 +41,10 @@ def _load():
         lib = C.CDLL(str(build()))
         lib.oracle_sam_build.restype = C.c_void_p
         lib.oracle_sam_build.argtypes = [_i32p, C.c_int64]
+        lib.oracle_sam_extend.restype = C.c_int
+        lib.oracle_sam_extend.argtypes = [C.c_void_p, _i32p, C.c_int64]
+        lib.oracle_renormalize.restype = C.c_int32
+        lib.oracle_renormalize.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         lib.oracle_sam_free.restype = None
         lib.oracle_sam_free.argtypes = [C.c_void_p]
         lib.oracle_sam_states.restype = C.c_int64
@@ -106,6 +110,20 @@ class OracleSAM:
         h, self.h = getattr(self, "h", None), None
         if h:
             self.lib.oracle_sam_free(h)
+
+    def extend(self, tokens) -> None:
+        """Appends tokens to the indexed text (the corpus copy used for drafting grows with it)."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        if self.lib.oracle_sam_extend(self.h, _i32(t), t.shape[0]):
+            raise MemoryError("oracle_sam_extend failed")
+        self.corpus = np.concatenate([self.corpus, t])
+        self.n = int(self.corpus.shape[0])
+
+    def renormalize(self, state, matched_len) -> None:
+        """In place: every (state[b], matched_len[b]) taken before the text grew is moved to the
+        state that now holds its string."""
+        for b in range(state.shape[0]):
+            state[b] = self.lib.oracle_renormalize(self.h, int(state[b]), int(matched_len[b]))
 
     @property
     def n_states(self) -> int:

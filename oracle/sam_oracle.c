@@ -53,6 +53,7 @@ typedef struct {
     ostate *st;
     int64_t n_states, cap_states;
     int64_t n_edges;
+    int64_t n_tokens;  /* corpus positions indexed so far */
     int32_t last;
 } osam;
 
@@ -159,6 +160,19 @@ void oracle_sam_free(osam *a)
     free(a);
 }
 
+/* Appends tokens[0..n) to the indexed text (Section 5.4.2: verified tokens are inserted into the
+ * automaton so that the index stays consistent with the growing context; Section 5.4.3: the
+ * construction is incremental, so appending is just more steps of it).  Returns 0, or -1 when out
+ * of memory. */
+int oracle_sam_extend(osam *a, const int32_t *tokens, int64_t n)
+{
+    for (int64_t i = 0; i < n; i++) {
+        if (extend(a, tokens[i], (int32_t)a->n_tokens)) return -1;
+        a->n_tokens++;
+    }
+    return 0;
+}
+
 /* Builds the automaton of corpus[0..n). Separators are ordinary symbols here. */
 osam *oracle_sam_build(const int32_t *corpus, int64_t n)
 {
@@ -172,10 +186,20 @@ osam *oracle_sam_build(const int32_t *corpus, int64_t n)
     a->st[root].link = -1;
     a->st[root].firstpos = -1;
     a->last = root;
-    for (int64_t i = 0; i < n; i++) {
-        if (extend(a, corpus[i], (int32_t)i)) { oracle_sam_free(a); return NULL; }
-    }
+    if (oracle_sam_extend(a, corpus, n)) { oracle_sam_free(a); return NULL; }
     return a;
+}
+
+/* A stream's pair (state, matched_len) taken before the automaton grew still names a string that
+ * occurs in the text, but a split may have moved that string into a new state: the state of a
+ * string of length L is the one with len(link(s)) < L <= len(s).  Climb suffix links until that
+ * holds again (the paper is silent on this; it follows from what the states of a suffix automaton
+ * are). */
+int32_t oracle_renormalize(const osam *a, int32_t state, int32_t matched_len)
+{
+    int32_t s = state;
+    while (s != 0 && matched_len <= a->st[a->st[s].link].len) s = a->st[s].link;
+    return s;
 }
 
 int64_t oracle_sam_states(const osam *a) { return a->n_states; }
