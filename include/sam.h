@@ -203,6 +203,59 @@ int sam_step_host(const sam_index* idx,
                   int32_t* next_drafts, int32_t* next_n_draft,
                   void* staging, int64_t staging_bytes, void* cuda_stream);
 
+/* ---------------------------------------------------------------- growing index */
+
+/* An index that keeps absorbing text after it was built (Section 5.4.2: verified tokens are
+ * inserted into the automaton so that it follows the growing context; Section 5.4.3 "Asynchronous
+ * SAM construction": building is handed to a child thread that serves a waiting queue, and
+ * drafting carries on with what is available until the new part is ready).
+ *
+ * sam_build_growing builds the automaton of corpus[0..n) (n may be 0) like sam_build, keeps the
+ * builder alive in a thread of its own, and sizes the device blob (sam_sizes) for up to max_tokens
+ * tokens: room for 2*max_tokens+2 state records, 6*max_tokens wide edges, a dense root table for token ids
+ * 0..max_token_id, the text, and an 8 MiB staging area for updates.  sam_upload, sam_draft,
+ * sam_verify, sam_step, sam_export, sam_sizes and sam_free work as for any other index.
+ *   max_tokens    1 .. 2^29, >= n;  max_token_id  largest token id that will ever be indexed
+ *                 (separators included), < 2^24
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOMEM. */
+int sam_build_growing(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep,
+                      int64_t max_tokens, int32_t max_token_id, sam_index** out);
+
+/* Appends tokens[0..n) (host) to the indexed text.  sam_extend_async copies them into the builder
+ * thread's queue and returns at once; sam_extend also waits until the builder thread has indexed
+ * everything queued so far.  Separators are appended like any other token (a new session is
+ * "SEP, tokens...").  Nothing changes on the device until sam_sync.
+ * Errors: SAM_ERR_INVALID_ARG (not a growing index, token id outside 0..max_token_id),
+ * SAM_ERR_TOO_LARGE (more than max_tokens in total), SAM_ERR_NOMEM. */
+int sam_extend_async(sam_index* idx, const int32_t* tokens, int64_t n);
+int sam_extend(sam_index* idx, const int32_t* tokens, int64_t n);
+
+/* Progress of a growing index, in tokens: handed in so far, indexed on the host so far, visible to
+ * the device kernels so far.  Any pointer may be NULL. */
+int sam_pending(sam_index* idx, int64_t* tokens_queued, int64_t* tokens_built, int64_t* tokens_on_device);
+
+/* Brings the device copy up to date with everything the builder thread has finished: the records
+ * of changed states, rewritten wide rows, changed root entries and the appended text are copied
+ * into the blob's staging area and scattered by small kernels on the stream (a whole new image is
+ * copied instead after the wide-edge area had to be laid out afresh).  Does not wait for the
+ * builder thread and does not synchronise the stream; hot-path calls enqueued afterwards on the
+ * same stream see the grown automaton.  Call it from the thread that makes the hot-path calls.
+ * After it, run sam_renormalize on every batch of stream states that will be used again.
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_TOO_LARGE (the automaton no longer
+ * fits the blob), SAM_ERR_CUDA. */
+int sam_sync(sam_index* idx, void* cuda_stream, int64_t* tokens_on_device);
+
+/* What sam_sync has applied to the device so far: updates that scattered only what changed, updates
+ * that copied a whole new image, and the host-to-device bytes of both.  Any pointer may be NULL. */
+int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_images, int64_t* bytes_copied);
+
+/* When the text grows, a state can be split, and a stream's (state, matched_len) may then name the
+ * half that no longer holds its string.  This moves every state[b] (device, [B], in place) up its
+ * suffix links to the state with len(link(s)) < matched_len[b] <= len(s); matched_len is unchanged.
+ * (The paper does not discuss this; it follows from what the states of a suffix automaton are.)
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_CUDA. */
+int sam_renormalize(const sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 
 /* Per-kernel device timing of sam_verify / sam_step (measurement aid; the paper has no

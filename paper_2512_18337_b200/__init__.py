@@ -10,6 +10,12 @@ from .binding import (  # noqa: F401
     exported_symbols,
     library_path,
     sam_build,
+    sam_build_growing,
+    sam_extend,
+    sam_pending,
+    sam_renormalize,
+    sam_sync,
+    sam_update_stats,
     sam_draft,
     sam_export,
     sam_free,

@@ -49,6 +49,13 @@ _SIGNATURES = {
     "sam_strerror": (C.c_char_p, [C.c_int]),
     "sam_last_cuda_error": (C.c_int, []),
     "sam_launch_count": (_i64, []),
+    "sam_build_growing": (C.c_int, [_vp, _i64, _vp, _i32, _i64, _i32, C.POINTER(_vp)]),
+    "sam_extend": (C.c_int, [_vp, _vp, _i64]),
+    "sam_extend_async": (C.c_int, [_vp, _vp, _i64]),
+    "sam_pending": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
+    "sam_sync": (C.c_int, [_vp, _vp, C.POINTER(_i64)]),
+    "sam_renormalize": (C.c_int, [_vp, _i32, _vp, _vp, _vp]),
+    "sam_update_stats": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
 }
 
 
@@ -130,6 +137,49 @@ def sam_build(corpus: np.ndarray, separators) -> int:
     _check(_load().sam_build(corpus.ctypes.data, corpus.shape[0], seps.ctypes.data if seps.size else None,
                              seps.shape[0], C.byref(h)), "sam_build")
     return h.value
+
+
+def sam_build_growing(corpus: np.ndarray, separators, max_tokens: int, max_token_id: int) -> int:
+    """Host build of an index that can grow (sam_extend); returns the opaque handle."""
+    corpus = np.ascontiguousarray(corpus, dtype=np.int32)
+    seps = np.ascontiguousarray(np.atleast_1d(separators), dtype=np.int32)
+    h = _vp()
+    _check(_load().sam_build_growing(corpus.ctypes.data if corpus.size else None, corpus.shape[0],
+                                     seps.ctypes.data if seps.size else None, seps.shape[0],
+                                     max_tokens, max_token_id, C.byref(h)), "sam_build_growing")
+    return h.value
+
+
+def sam_extend(handle: int, tokens: np.ndarray, wait: bool = True) -> None:
+    """Appends host tokens; wait=False only queues them for the builder thread (sam_extend_async)."""
+    t = np.ascontiguousarray(tokens, dtype=np.int32)
+    fn = _load().sam_extend if wait else _load().sam_extend_async
+    _check(fn(handle, t.ctypes.data if t.size else None, t.shape[0]), "sam_extend" if wait else "sam_extend_async")
+
+
+def sam_pending(handle: int):
+    """(tokens_queued, tokens_built, tokens_on_device)."""
+    a, b, c = _i64(), _i64(), _i64()
+    _check(_load().sam_pending(handle, C.byref(a), C.byref(b), C.byref(c)), "sam_pending")
+    return a.value, b.value, c.value
+
+
+def sam_sync(handle: int, stream=None) -> int:
+    """Applies finished updates to the device copy; returns the tokens visible on the device."""
+    n = _i64()
+    _check(_load().sam_sync(handle, _stream(stream), C.byref(n)), "sam_sync")
+    return int(n.value)
+
+
+def sam_update_stats(handle: int):
+    """(incremental updates, whole-image updates, bytes copied) applied by sam_sync so far."""
+    a, b, c = _i64(), _i64(), _i64()
+    _check(_load().sam_update_stats(handle, C.byref(a), C.byref(b), C.byref(c)), "sam_update_stats")
+    return a.value, b.value, c.value
+
+
+def sam_renormalize(handle: int, B: int, state, matched_len, stream=None) -> None:
+    _check(_load().sam_renormalize(handle, B, _dev(state), _dev(matched_len), _stream(stream)), "sam_renormalize")
 
 
 def sam_sizes(handle: int):
@@ -272,8 +322,13 @@ def sam_launch_count() -> int:
 class SamIndex:
     """Owns a built handle and the torch tensor that holds its device blob (memory plumbing only)."""
 
-    def __init__(self, corpus: np.ndarray, separators, device="cuda:0", upload: bool = True):
-        self.handle = sam_build(corpus, separators)
+    def __init__(self, corpus: np.ndarray, separators, device="cuda:0", upload: bool = True,
+                 max_tokens: Optional[int] = None, max_token_id: Optional[int] = None):
+        """max_tokens given: an index that can grow up to that many tokens (sam_build_growing)."""
+        if max_tokens is None:
+            self.handle = sam_build(corpus, separators)
+        else:
+            self.handle = sam_build_growing(corpus, separators, max_tokens, max_token_id)
         self.n_states, self.n_edges, self.device_bytes = sam_sizes(self.handle)
         self.blob = None
         if upload:

@@ -9,8 +9,8 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libsam_b200.so"
-SOURCES = [CSRC / "sam_capi.cu", CSRC / "sam_build.cpp"]
-HEADERS = [ROOT / "include" / "sam.h", CSRC / "sam_index.h", CSRC / "sam_kernels.cuh", CSRC / "argmax_bulk.cuh"]
+SOURCES = [CSRC / "sam_capi.cu", CSRC / "sam_build.cpp", CSRC / "sam_dynamic.cpp"]
+HEADERS = [ROOT / "include" / "sam.h"] + sorted(CSRC.glob("*.h")) + sorted(CSRC.glob("*.cuh"))
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -13,6 +13,7 @@
 #include "sam_index.h"
 #include "sam_kernels.cuh"
 #include "argmax_bulk.cuh"
+#include "sam_update.cuh"
 
 using namespace samb200;
 
@@ -188,6 +189,147 @@ int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st) {
     return SAM_OK;
 }
 
+// ---- growing index: device side of an update ---------------------------------------------------
+void set_device_view(sam_index* idx, void* device_buf) {
+    const DeviceLayout& L = idx->layout;
+    char* base = static_cast<char*>(device_buf);
+    DeviceSam& d = idx->dev;
+    d.rec = reinterpret_cast<const StateRec*>(base + L.rec_off);
+    d.wide = reinterpret_cast<const Edge*>(base + L.edge_off);
+    d.root_dst = reinterpret_cast<const int32_t*>(base + L.root_off);
+    d.corpus = reinterpret_cast<const int32_t*>(base + L.corpus_off);
+    d.root_span = static_cast<int32_t>(L.root_span);
+    d.n_sep = static_cast<int32_t>(idx->seps.size());
+    for (int k = 0; k < SAM_MAX_SEPARATORS; ++k) d.seps[k] = (k < d.n_sep) ? idx->seps[k] : -1;
+}
+
+// Copies a whole image (first upload, or after the wide rows were laid out afresh).
+int apply_full(sam_index* idx, const Delta& D, cudaStream_t st) {
+    const DeviceLayout& L = idx->layout;
+    char* base = static_cast<char*>(idx->device_buf);
+    SAM_CUDA(cudaMemcpyAsync(base + L.rec_off, D.all_rec.data(), D.all_rec.size() * sizeof(StateRec), cudaMemcpyHostToDevice, st));
+    if (!D.all_wide.empty())
+        SAM_CUDA(cudaMemcpyAsync(base + L.edge_off, D.all_wide.data(), D.all_wide.size() * sizeof(Edge), cudaMemcpyHostToDevice, st));
+    SAM_CUDA(cudaMemcpyAsync(base + L.root_off, D.all_root.data(), D.all_root.size() * 4, cudaMemcpyHostToDevice, st));
+    if (!D.all_corpus.empty())
+        SAM_CUDA(cudaMemcpyAsync(base + L.corpus_off, D.all_corpus.data(), D.all_corpus.size() * 4, cudaMemcpyHostToDevice, st));
+    return SAM_OK;
+}
+
+constexpr int kDirectRowEdges = 2048;   // rows at least this long are copied straight to their place
+
+// Scatters one update through the staging area, in as many rounds as its size needs.  Host buffers are
+// pageable, so every cudaMemcpyAsync has taken its copy of the source when it returns.
+int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st) {
+    const DeviceLayout& L = idx->layout;
+    char* base = static_cast<char*>(idx->device_buf);
+    char* stage = base + L.stage_off;
+    StateRec* rec = reinterpret_cast<StateRec*>(base + L.rec_off);
+    Edge* wide = reinterpret_cast<Edge*>(base + L.edge_off);
+    int32_t* root = reinterpret_cast<int32_t*>(base + L.root_off);
+    std::vector<char> buf;
+    // records: [ids (padded to 32 B)] [records]
+    const int64_t n_rec = static_cast<int64_t>(D.rec_ids.size());
+    const int64_t per_round = (L.stage_bytes - 64) / 36;
+    for (int64_t i0 = 0; i0 < n_rec; i0 += per_round) {
+        const int64_t n = std::min(per_round, n_rec - i0);
+        const int64_t ids_bytes = (n * 4 + 31) & ~int64_t(31);
+        buf.resize(static_cast<size_t>(ids_bytes + n * 32));
+        std::memcpy(buf.data(), D.rec_ids.data() + i0, static_cast<size_t>(n) * 4);
+        std::memcpy(buf.data() + ids_bytes, D.recs.data() + i0, static_cast<size_t>(n) * 32);
+        SAM_CUDA(cudaMemcpyAsync(stage, buf.data(), buf.size(), cudaMemcpyHostToDevice, st));
+        scatter_records_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+            rec, reinterpret_cast<const int32_t*>(stage), reinterpret_cast<const StateRec*>(stage + ids_bytes),
+            static_cast<int>(n));
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+    }
+    // wide rows: long ones directly, short ones in batches of [descriptors] [edges]
+    std::vector<SegDesc> descs;
+    std::vector<Edge> edges;
+    auto flush_rows = [&]() -> int {
+        if (descs.empty()) return SAM_OK;
+        const int64_t d_bytes = (static_cast<int64_t>(descs.size()) * sizeof(SegDesc) + 31) & ~int64_t(31);
+        buf.resize(static_cast<size_t>(d_bytes) + edges.size() * sizeof(Edge));
+        std::memcpy(buf.data(), descs.data(), descs.size() * sizeof(SegDesc));
+        std::memcpy(buf.data() + d_bytes, edges.data(), edges.size() * sizeof(Edge));
+        SAM_CUDA(cudaMemcpyAsync(stage, buf.data(), buf.size(), cudaMemcpyHostToDevice, st));
+        const int n = static_cast<int>(descs.size());
+        copy_rows_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(
+            wide, reinterpret_cast<const SegDesc*>(stage), reinterpret_cast<const Edge*>(stage + d_bytes), n);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+        descs.clear();
+        edges.clear();
+        return SAM_OK;
+    };
+    for (const WideSeg& g : D.segs) {
+        if (g.len >= kDirectRowEdges) {
+            SAM_CUDA(cudaMemcpyAsync(wide + g.dst_off, D.seg_edges.data() + g.src_off, static_cast<size_t>(g.len) * sizeof(Edge),
+                                     cudaMemcpyHostToDevice, st));
+            continue;
+        }
+        const int64_t need = (static_cast<int64_t>(descs.size()) + 1) * sizeof(SegDesc) + 32 +
+                             (static_cast<int64_t>(edges.size()) + g.len) * sizeof(Edge);
+        if (need > L.stage_bytes) {
+            const int rc = flush_rows();
+            if (rc != SAM_OK) return rc;
+        }
+        descs.push_back(SegDesc{g.dst_off, static_cast<int>(edges.size()), g.len});
+        edges.insert(edges.end(), D.seg_edges.begin() + g.src_off, D.seg_edges.begin() + g.src_off + g.len);
+    }
+    {
+        const int rc = flush_rows();
+        if (rc != SAM_OK) return rc;
+    }
+    // root entries: [tokens (padded)] [destinations]
+    const int64_t n_root = static_cast<int64_t>(D.root_tok.size());
+    const int64_t root_round = (L.stage_bytes - 64) / 8;
+    for (int64_t i0 = 0; i0 < n_root; i0 += root_round) {
+        const int64_t n = std::min(root_round, n_root - i0);
+        const int64_t t_bytes = (n * 4 + 31) & ~int64_t(31);
+        buf.resize(static_cast<size_t>(t_bytes + n * 4));
+        std::memcpy(buf.data(), D.root_tok.data() + i0, static_cast<size_t>(n) * 4);
+        std::memcpy(buf.data() + t_bytes, D.root_dst.data() + i0, static_cast<size_t>(n) * 4);
+        SAM_CUDA(cudaMemcpyAsync(stage, buf.data(), buf.size(), cudaMemcpyHostToDevice, st));
+        scatter_root_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+            root, reinterpret_cast<const int32_t*>(stage), reinterpret_cast<const int32_t*>(stage + t_bytes),
+            static_cast<int>(n), static_cast<int>(L.root_span));
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+    }
+    if (!D.corpus_tail.empty())
+        SAM_CUDA(cudaMemcpyAsync(base + L.corpus_off + D.corpus_off * 4, D.corpus_tail.data(), D.corpus_tail.size() * 4,
+                                 cudaMemcpyHostToDevice, st));
+    return SAM_OK;
+}
+
+int apply_delta(sam_index* idx, const Delta& D, cudaStream_t st) {
+    if (D.status != SAM_OK) return D.status;
+    const int rc = D.full ? apply_full(idx, D, st) : apply_changes(idx, D, st);
+    if (rc != SAM_OK) return rc;
+    idx->dev.n_states = static_cast<int32_t>(D.n_states_after);
+    idx->dev.n_corpus = D.n_tokens_after;
+    idx->layout.n_states = D.n_states_after;
+    idx->layout.n_corpus = D.n_tokens_after;
+    return SAM_OK;
+}
+
+int upload_growing(sam_index* idx, void* device_buf, cudaStream_t st) {
+    Delta image;
+    int rc = dyn_full_image(idx, &image);
+    if (rc != SAM_OK) return rc;
+    idx->device_buf = device_buf;
+    set_device_view(idx, device_buf);
+    rc = apply_delta(idx, image, st);
+    if (rc != SAM_OK) {
+        idx->device_buf = nullptr;
+        return rc;
+    }
+    SAM_CUDA(cudaStreamSynchronize(st));
+    return SAM_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -210,6 +352,11 @@ int sam_build(const int32_t* corpus, int64_t n, const int32_t* separators, int32
 
 int sam_sizes(const sam_index* idx, int64_t* n_states, int64_t* n_edges, int64_t* device_bytes) {
     if (!idx) return SAM_ERR_INVALID_ARG;
+    if (idx->dyn) {
+        const int rc = dyn_sizes(const_cast<sam_index*>(idx), n_states, n_edges);
+        if (device_bytes) *device_bytes = idx->layout.total;
+        return rc;
+    }
     if (n_states) *n_states = idx->layout.n_states;
     if (n_edges) *n_edges = static_cast<int64_t>(idx->edge_tok.size());
     if (device_bytes) *device_bytes = idx->layout.total;
@@ -219,6 +366,10 @@ int sam_sizes(const sam_index* idx, int64_t* n_states, int64_t* n_edges, int64_t
 int sam_export(const sam_index* idx, int32_t* len, int32_t* link, int32_t* firstpos,
                int64_t* row_ptr, int32_t* edge_tok, int32_t* edge_dst) {
     if (!idx) return SAM_ERR_INVALID_ARG;
+    if (idx->dyn) {
+        const int rc = dyn_refresh_csr(const_cast<sam_index*>(idx));
+        if (rc != SAM_OK) return rc;
+    }
     const size_t S = idx->len.size(), E = idx->edge_tok.size();
     if (len) std::memcpy(len, idx->len.data(), S * 4);
     if (link) std::memcpy(link, idx->link.data(), S * 4);
@@ -234,6 +385,7 @@ int sam_upload(sam_index* idx, void* device_buf, int64_t bytes, void* cuda_strea
     const DeviceLayout& L = idx->layout;
     if (bytes < L.total) return SAM_ERR_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (idx->dyn) return upload_growing(idx, device_buf, st);
     std::vector<StateRec> rec;
     std::vector<Edge> wide;
     std::vector<int32_t> root;
@@ -267,7 +419,11 @@ int sam_upload(sam_index* idx, void* device_buf, int64_t bytes, void* cuda_strea
     return SAM_OK;
 }
 
-void sam_free(sam_index* idx) { delete idx; }
+void sam_free(sam_index* idx) {
+    if (!idx) return;
+    dyn_destroy(idx);
+    delete idx;
+}
 
 int64_t sam_workspace_bytes(int32_t B, int32_t K) {
     if (B < 0 || K < 1 || K > SAM_K_MAX) return SAM_ERR_INVALID_ARG;
@@ -482,6 +638,86 @@ int sam_step_host(const sam_index* idx,
     SAM_CUDA(cudaMemcpyAsync(next_drafts, d + L.drafts, bK, cudaMemcpyDeviceToHost, st));
     SAM_CUDA(cudaMemcpyAsync(next_n_draft, d + L.n_draft, bB, cudaMemcpyDeviceToHost, st));
     SAM_CUDA(cudaStreamSynchronize(st));
+    return SAM_OK;
+}
+
+int sam_build_growing(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep,
+                      int64_t max_tokens, int32_t max_token_id, sam_index** out) {
+    if (!out || n < 0 || (n > 0 && !corpus)) return SAM_ERR_INVALID_ARG;
+    if (n_sep < 0 || n_sep > SAM_MAX_SEPARATORS || (n_sep > 0 && !separators)) return SAM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; ++i)
+        if (corpus[i] < 0) return SAM_ERR_INVALID_ARG;
+    sam_index* idx = new (std::nothrow) sam_index();
+    if (!idx) return SAM_ERR_NOMEM;
+    idx->seps.assign(separators, separators + n_sep);
+    const int rc = dyn_create(idx, corpus, n, max_tokens, max_token_id);
+    if (rc != SAM_OK) {
+        delete idx;
+        return rc;
+    }
+    *out = idx;
+    return SAM_OK;
+}
+
+int sam_extend_async(sam_index* idx, const int32_t* tokens, int64_t n) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    return dyn_enqueue(idx, tokens, n);
+}
+
+int sam_extend(sam_index* idx, const int32_t* tokens, int64_t n) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    const int rc = dyn_enqueue(idx, tokens, n);
+    if (rc != SAM_OK) return rc;
+    return dyn_wait(idx);
+}
+
+int sam_pending(sam_index* idx, int64_t* tokens_queued, int64_t* tokens_built, int64_t* tokens_on_device) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    dyn_counts(idx, tokens_queued, tokens_built);
+    if (tokens_on_device) *tokens_on_device = idx->device_buf ? idx->dev.n_corpus : 0;
+    return SAM_OK;
+}
+
+int sam_sync(sam_index* idx, void* cuda_stream, int64_t* tokens_on_device) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Delta D;
+    while (dyn_pop_ready(idx, &D)) {
+        const int rc = apply_delta(idx, D, st);
+        if (rc != SAM_OK) return rc;
+        if (D.full) {
+            ++idx->updates_full;
+            idx->update_bytes += static_cast<int64_t>(D.all_rec.size() * sizeof(StateRec) + D.all_wide.size() * sizeof(Edge) +
+                                                      (D.all_root.size() + D.all_corpus.size()) * 4);
+        } else {
+            ++idx->updates_incremental;
+            idx->update_bytes += static_cast<int64_t>(D.rec_ids.size() * 36 + D.seg_edges.size() * sizeof(Edge) +
+                                                      D.segs.size() * sizeof(SegDesc) + D.root_tok.size() * 8 +
+                                                      D.corpus_tail.size() * 4);
+        }
+    }
+    if (tokens_on_device) *tokens_on_device = idx->dev.n_corpus;
+    return SAM_OK;
+}
+
+int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_images, int64_t* bytes_copied) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    if (incremental) *incremental = idx->updates_incremental;
+    if (full_images) *full_images = idx->updates_full;
+    if (bytes_copied) *bytes_copied = idx->update_bytes;
+    return SAM_OK;
+}
+
+int sam_renormalize(const sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream) {
+    if (!idx || B < 0) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!state || !matched_len) return SAM_ERR_INVALID_ARG;
+    renormalize_kernel<<<static_cast<unsigned>((B + 127) / 128), 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        idx->dev, B, state, matched_len);
+    SAM_CUDA(cudaGetLastError());
+    ++g_launches;
     return SAM_OK;
 }
 

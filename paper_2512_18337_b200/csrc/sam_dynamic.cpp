@@ -1,0 +1,366 @@
+// Growing index: the automaton keeps absorbing tokens after it was built (Section 5.4.2: verified
+// tokens are inserted so that the index follows the growing context) and a builder thread does the
+// construction off the decoding path (Section 5.4.3: construction is offloaded to a child thread
+// that serves a waiting queue; until an update is ready, drafting goes on with what is there).
+//
+// The builder thread owns the automaton.  For every chunk of tokens it takes from the queue it runs
+// the online construction, then packs what changed - records of touched states, rewritten wide
+// rows, changed root entries, the appended text - into a Delta that the caller's thread later
+// copies to the device (sam_sync).  Wide rows get power-of-two capacity so that most rewrites happen
+// in place; when the wide area is exhausted all rows are laid out afresh and the next update is a
+// full image.
+#include <algorithm>
+#include <condition_variable>
+#include <cstdlib>
+#include <cstring>
+#include <deque>
+#include <mutex>
+#include <new>
+#include <thread>
+#include <unordered_map>
+
+#include "sam_builder.h"
+#include "sam_index.h"
+
+namespace samb200 {
+
+struct DynIndex {
+    Builder b;
+    int32_t last = 0;
+    std::vector<int32_t> corpus;
+    int64_t max_tokens = 0, s_cap = 0, w_cap = 0, span_cap = 0;
+    std::vector<int32_t> wide_off, wide_cap;   // per state: row offset / capacity in the device's wide array (-1 / 0: none)
+    int64_t w_used = 0;
+
+    std::thread worker;
+    std::mutex mu;
+    std::condition_variable cv_work, cv_idle;
+    std::deque<std::vector<int32_t>> inbox;
+    std::deque<Delta> ready;
+    bool stop = false, busy = false;
+    int64_t queued = 0, built = 0;
+    int error = SAM_OK;
+};
+
+namespace {
+
+int32_t pow2_at_least(int32_t d) {
+    int32_t c = 4;
+    while (c < d) c <<= 1;
+    return c;
+}
+
+// Record of state s (not the root); a wide row is placed (or re-placed) when it outgrew its slot.
+// Returns false when the wide area is exhausted.
+bool pack_state(DynIndex& D, int32_t s, StateRec* r, std::vector<std::pair<int32_t, int32_t>>& row, bool* is_wide) {
+    const Builder& b = D.b;
+    r->len = b.len[s];
+    r->link = b.link[s];
+    r->firstpos = b.fpos[s];
+    r->deg = b.deg[s];
+    r->e[0] = r->e[1] = r->e[2] = r->e[3] = -1;
+    b.sorted_row(s, row);
+    const int32_t d = b.deg[s];
+    *is_wide = d >= 3;
+    if (d >= 1 && d <= 2) {
+        r->e[0] = row[0].first;
+        r->e[1] = row[0].second;
+        if (d == 2) { r->e[2] = row[1].first; r->e[3] = row[1].second; }
+    } else if (d >= 3) {
+        if (static_cast<size_t>(s) >= D.wide_off.size()) {
+            D.wide_off.resize(b.len.size(), -1);
+            D.wide_cap.resize(b.len.size(), 0);
+        }
+        if (D.wide_cap[s] < d) {
+            const int32_t cap = pow2_at_least(d);
+            if (D.w_used + cap > D.w_cap) return false;
+            D.wide_off[s] = static_cast<int32_t>(D.w_used);
+            D.wide_cap[s] = cap;
+            D.w_used += cap;
+        }
+        r->e[0] = D.wide_off[s];
+    }
+    return true;
+}
+
+// Everything, laid out afresh (wide rows compacted).
+int pack_full(DynIndex& D, Delta* out) {
+    const Builder& b = D.b;
+    const int64_t S = static_cast<int64_t>(b.len.size());
+    out->full = true;
+    out->all_rec.assign(static_cast<size_t>(S), StateRec{});
+    out->all_root.assign(static_cast<size_t>(D.span_cap), -1);
+    D.wide_off.assign(static_cast<size_t>(S), -1);
+    D.wide_cap.assign(static_cast<size_t>(S), 0);
+    D.w_used = 0;
+    std::vector<std::pair<int32_t, int32_t>> row;
+    // first pass places the rows, second copies them (the total is known only after placing)
+    for (int64_t s = 1; s < S; ++s) {
+        bool wide = false;
+        if (!pack_state(D, static_cast<int32_t>(s), &out->all_rec[s], row, &wide)) return SAM_ERR_TOO_LARGE;
+    }
+    out->all_wide.assign(static_cast<size_t>(D.w_used), Edge{-1, -1});
+    for (int64_t s = 1; s < S; ++s) {
+        if (b.deg[s] < 3) continue;
+        b.sorted_row(static_cast<int32_t>(s), row);
+        Edge* dst = out->all_wide.data() + D.wide_off[s];
+        for (size_t k = 0; k < row.size(); ++k) dst[k] = Edge{row[k].first, row[k].second};
+    }
+    StateRec& r0 = out->all_rec[0];
+    r0.len = 0; r0.link = -1; r0.firstpos = -1; r0.deg = b.deg[0];
+    r0.e[0] = r0.e[1] = r0.e[2] = r0.e[3] = -1;
+    for (int32_t x = b.head[0]; x >= 0; x = b.e_next[x]) out->all_root[b.e_tok[x]] = b.e_dst[x];
+    out->all_corpus = D.corpus;
+    out->n_states_after = S;
+    out->n_tokens_after = static_cast<int64_t>(D.corpus.size());
+    return SAM_OK;
+}
+
+// What the last chunk changed.
+int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
+    Builder& b = D.b;
+    std::vector<std::pair<int32_t, int32_t>> row;
+    out->rec_ids.reserve(b.dirty.size());
+    out->recs.reserve(b.dirty.size());
+    for (int32_t s : b.dirty) {
+        StateRec r;
+        bool wide = false;
+        if (!pack_state(D, s, &r, row, &wide)) {
+            // wide area exhausted: lay everything out afresh and send the whole image instead
+            Delta fresh;
+            const int rc = pack_full(D, &fresh);
+            *out = std::move(fresh);
+            return rc;
+        }
+        out->rec_ids.push_back(s);
+        out->recs.push_back(r);
+        if (wide) {
+            WideSeg g;
+            g.dst_off = D.wide_off[s];
+            g.src_off = static_cast<int64_t>(out->seg_edges.size());
+            g.len = static_cast<int32_t>(row.size());
+            out->segs.push_back(g);
+            for (const auto& e : row) out->seg_edges.push_back(Edge{e.first, e.second});
+        }
+    }
+    // root: the last change of a token wins
+    std::unordered_map<int32_t, int32_t> last;
+    last.reserve(b.root_changes.size() * 2 + 1);
+    for (const auto& c : b.root_changes) last[c.first] = c.second;
+    out->root_tok.reserve(last.size());
+    out->root_dst.reserve(last.size());
+    for (const auto& kv : last) { out->root_tok.push_back(kv.first); out->root_dst.push_back(kv.second); }
+    out->corpus_off = corpus_before;
+    out->corpus_tail.assign(D.corpus.begin() + corpus_before, D.corpus.end());
+    out->n_states_after = static_cast<int64_t>(b.len.size());
+    out->n_tokens_after = static_cast<int64_t>(D.corpus.size());
+    return SAM_OK;
+}
+
+void worker_main(DynIndex* D) {
+    for (;;) {
+        std::vector<int32_t> chunk;
+        {
+            std::unique_lock<std::mutex> lk(D->mu);
+            D->cv_work.wait(lk, [&] { return D->stop || !D->inbox.empty(); });
+            if (D->stop) return;
+            chunk.swap(D->inbox.front());
+            D->inbox.pop_front();
+            D->busy = true;
+        }
+        Delta delta;
+        int rc = SAM_OK;
+        try {
+            const int64_t before = static_cast<int64_t>(D->corpus.size());
+            for (int32_t c : chunk) {
+                D->b.extend(c, static_cast<int32_t>(D->corpus.size()), D->last);
+                D->corpus.push_back(c);
+            }
+            rc = pack_changes(*D, before, &delta);
+            D->b.clear_changes();
+        } catch (const std::bad_alloc&) {
+            rc = SAM_ERR_NOMEM;
+        }
+        delta.status = rc;
+        {
+            std::lock_guard<std::mutex> lk(D->mu);
+            if (rc != SAM_OK) D->error = rc;
+            D->built += static_cast<int64_t>(chunk.size());
+            D->ready.push_back(std::move(delta));
+            D->busy = false;
+        }
+        D->cv_idle.notify_all();
+    }
+}
+
+}  // namespace
+
+int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tokens, int32_t max_token_id) {
+    if (max_tokens < n || max_tokens < 1 || max_tokens > (int64_t(1) << 29) || max_token_id < 0 ||
+        max_token_id >= (1 << 24))
+        return SAM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; ++i)
+        if (corpus[i] > max_token_id) return SAM_ERR_INVALID_ARG;
+    DynIndex* D = nullptr;
+    try {
+        D = new DynIndex();
+        D->max_tokens = max_tokens;
+        D->s_cap = 2 * max_tokens + 2;
+        // rows hold at most 3N transitions in total and a row's slot is less than twice its length, so a fresh
+        // layout always fits 6N; the rest of the area absorbs rows that outgrew their slot
+        double per_token = 6.0;
+        if (const char* e = std::getenv("SAM_B200_WIDE_EDGES_PER_TOKEN")) {   // tuning / test knob
+            const double v = std::atof(e);
+            if (v >= 0.25 && v <= 64.0) per_token = v;
+        }
+        D->w_cap = std::min<int64_t>(static_cast<int64_t>(per_token * static_cast<double>(max_tokens)) + 1024,
+                                     (int64_t(1) << 31) - 64);
+        D->span_cap = static_cast<int64_t>(max_token_id) + 1;
+        Builder& b = D->b;
+        b.hash_alloc(1u << 16);
+        b.new_state(0, -1, -1);
+        D->corpus.reserve(static_cast<size_t>(std::min<int64_t>(max_tokens, n + (int64_t(1) << 20))));
+        for (int64_t i = 0; i < n; ++i) {
+            b.extend(corpus[i], static_cast<int32_t>(i), D->last);
+            D->corpus.push_back(corpus[i]);
+        }
+        b.track = true;
+        b.mark.assign(b.len.size(), 0);
+        D->queued = D->built = n;
+    } catch (const std::bad_alloc&) {
+        delete D;
+        return SAM_ERR_NOMEM;
+    }
+    auto up = [](int64_t x) { return (x + 255) & ~int64_t(255); };
+    DeviceLayout& L = idx->layout;
+    L.n_states = static_cast<int64_t>(D->b.len.size());
+    L.n_corpus = n;
+    L.root_span = D->span_cap;
+    L.n_wide_edges = D->w_cap;
+    L.stage_bytes = int64_t(8) << 20;
+    L.rec_off = 0;
+    L.edge_off = up(L.rec_off + D->s_cap * static_cast<int64_t>(sizeof(StateRec)));
+    L.root_off = up(L.edge_off + D->w_cap * static_cast<int64_t>(sizeof(Edge)));
+    L.corpus_off = up(L.root_off + D->span_cap * 4);
+    L.stage_off = up(L.corpus_off + max_tokens * 4);
+    L.total = up(L.stage_off + L.stage_bytes);
+    idx->dyn = D;
+    D->worker = std::thread(worker_main, D);
+    return SAM_OK;
+}
+
+void dyn_destroy(sam_index* idx) {
+    DynIndex* D = idx->dyn;
+    if (!D) return;
+    {
+        std::lock_guard<std::mutex> lk(D->mu);
+        D->stop = true;
+    }
+    D->cv_work.notify_all();
+    if (D->worker.joinable()) D->worker.join();
+    delete D;
+    idx->dyn = nullptr;
+}
+
+int dyn_enqueue(sam_index* idx, const int32_t* tokens, int64_t n) {
+    DynIndex* D = idx->dyn;
+    if (!D || n < 0 || (n > 0 && !tokens)) return SAM_ERR_INVALID_ARG;
+    if (n == 0) return SAM_OK;
+    for (int64_t i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= D->span_cap) return SAM_ERR_INVALID_ARG;
+    {
+        std::lock_guard<std::mutex> lk(D->mu);
+        if (D->error != SAM_OK) return D->error;
+        if (D->queued + n > D->max_tokens) return SAM_ERR_TOO_LARGE;
+        try {
+            D->inbox.emplace_back(tokens, tokens + n);
+        } catch (const std::bad_alloc&) {
+            return SAM_ERR_NOMEM;
+        }
+        D->queued += n;
+    }
+    D->cv_work.notify_one();
+    return SAM_OK;
+}
+
+int dyn_wait(sam_index* idx) {
+    DynIndex* D = idx->dyn;
+    if (!D) return SAM_ERR_INVALID_ARG;
+    std::unique_lock<std::mutex> lk(D->mu);
+    D->cv_idle.wait(lk, [&] { return D->inbox.empty() && !D->busy; });
+    return D->error;
+}
+
+bool dyn_pop_ready(sam_index* idx, Delta* out) {
+    DynIndex* D = idx->dyn;
+    std::lock_guard<std::mutex> lk(D->mu);
+    if (D->ready.empty()) return false;
+    *out = std::move(D->ready.front());
+    D->ready.pop_front();
+    return true;
+}
+
+int dyn_full_image(sam_index* idx, Delta* out) {
+    DynIndex* D = idx->dyn;
+    if (!D) return SAM_ERR_INVALID_ARG;
+    std::unique_lock<std::mutex> lk(D->mu);
+    D->cv_idle.wait(lk, [&] { return D->inbox.empty() && !D->busy; });
+    D->ready.clear();            // whatever they held is part of the image
+    try {
+        return pack_full(*D, out);
+    } catch (const std::bad_alloc&) {
+        return SAM_ERR_NOMEM;
+    }
+}
+
+int dyn_refresh_csr(sam_index* idx) {
+    DynIndex* D = idx->dyn;
+    if (!D) return SAM_ERR_INVALID_ARG;
+    std::unique_lock<std::mutex> lk(D->mu);
+    D->cv_idle.wait(lk, [&] { return D->inbox.empty() && !D->busy; });
+    try {
+        const Builder& b = D->b;
+        const size_t S = b.len.size(), E = b.e_tok.size();
+        idx->len = b.len;
+        idx->link = b.link;
+        idx->firstpos = b.fpos;
+        idx->row_ptr.resize(S + 1);
+        idx->edge_tok.resize(E);
+        idx->edge_dst.resize(E);
+        std::vector<std::pair<int32_t, int32_t>> row;
+        int64_t off = 0;
+        for (size_t s = 0; s < S; ++s) {
+            idx->row_ptr[s] = off;
+            b.sorted_row(static_cast<int32_t>(s), row);
+            for (const auto& e : row) {
+                idx->edge_tok[off] = e.first;
+                idx->edge_dst[off] = e.second;
+                ++off;
+            }
+        }
+        idx->row_ptr[S] = off;
+        idx->layout.n_states = static_cast<int64_t>(S);
+    } catch (const std::bad_alloc&) {
+        return SAM_ERR_NOMEM;
+    }
+    return SAM_OK;
+}
+
+int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges) {
+    DynIndex* D = idx->dyn;
+    if (!D) return SAM_ERR_INVALID_ARG;
+    std::unique_lock<std::mutex> lk(D->mu);
+    D->cv_idle.wait(lk, [&] { return D->inbox.empty() && !D->busy; });
+    if (n_states) *n_states = static_cast<int64_t>(D->b.len.size());
+    if (n_edges) *n_edges = static_cast<int64_t>(D->b.e_tok.size());
+    return SAM_OK;
+}
+
+void dyn_counts(sam_index* idx, int64_t* queued, int64_t* built) {
+    DynIndex* D = idx->dyn;
+    std::lock_guard<std::mutex> lk(D->mu);
+    if (queued) *queued = D->queued;
+    if (built) *built = D->built;
+}
+
+}  // namespace samb200

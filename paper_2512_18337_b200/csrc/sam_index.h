@@ -21,9 +21,10 @@ static_assert(sizeof(StateRec) == 32, "one sector per state");
 struct Edge { int32_t tok, dst; };  // wide rows: ascending by tok
 
 // Where things sit inside the caller's device blob (byte offsets, 256-byte aligned).
+// A growing index sizes every section for its capacity and adds a staging area for updates.
 struct DeviceLayout {
-    int64_t rec_off = 0, edge_off = 0, root_off = 0, corpus_off = 0, total = 0;
-    int64_t n_states = 0, n_wide_edges = 0, root_span = 0, n_corpus = 0;
+    int64_t rec_off = 0, edge_off = 0, root_off = 0, corpus_off = 0, stage_off = 0, total = 0;
+    int64_t n_states = 0, n_wide_edges = 0, root_span = 0, n_corpus = 0, stage_bytes = 0;
 };
 
 // Pointers handed to kernels by value.
@@ -40,6 +41,31 @@ struct DeviceSam {
     int32_t seps[SAM_MAX_SEPARATORS];
 };
 
+// ---- growing index (appending verified tokens; Section 5.4.2 / 5.4.3) --------------------------
+// What changed on the host since the device image was last brought up to date.
+struct WideSeg {
+    int64_t dst_off;   // first edge of the row in the device's wide array
+    int64_t src_off;   // first edge of the row in Delta::seg_edges
+    int32_t len;
+};
+struct Delta {
+    bool full = false;                       // whole image (first upload, or after the wide rows were compacted)
+    int status = SAM_OK;
+    std::vector<int32_t> rec_ids;            // states whose 32-byte record changed ...
+    std::vector<StateRec> recs;              // ... and the new records
+    std::vector<WideSeg> segs;               // wide rows to (re)write
+    std::vector<Edge> seg_edges;
+    std::vector<int32_t> root_tok, root_dst; // changed entries of the dense root table (one per token)
+    int64_t corpus_off = 0;                  // appended text
+    std::vector<int32_t> corpus_tail;
+    int64_t n_states_after = 0, n_tokens_after = 0;
+    // full image only
+    std::vector<StateRec> all_rec;
+    std::vector<Edge> all_wide;
+    std::vector<int32_t> all_root, all_corpus;
+};
+struct DynIndex;   // host-side state of a growing index (sam_dynamic.cpp)
+
 }  // namespace samb200
 
 struct sam_index {
@@ -53,6 +79,9 @@ struct sam_index {
     // set by sam_upload
     void* device_buf = nullptr;
     samb200::DeviceSam dev{};
+    // growing index only
+    samb200::DynIndex* dyn = nullptr;
+    int64_t updates_incremental = 0, updates_full = 0, update_bytes = 0;   // what sam_sync has applied so far
 };
 
 namespace samb200 {
@@ -60,4 +89,15 @@ namespace samb200 {
 int build_index(const int32_t* corpus, int64_t n, const int32_t* seps, int32_t n_sep, sam_index* out);
 // Fills the packed host image of the device blob (rec / wide edges / root table); corpus is copied separately.
 void pack_records(const sam_index& idx, StateRec* rec, Edge* wide, int32_t* root_dst);
+
+// Growing index.  All of these are host-side; none touches the device.
+int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tokens, int32_t max_token_id);
+void dyn_destroy(sam_index* idx);
+int dyn_enqueue(sam_index* idx, const int32_t* tokens, int64_t n);     // hands tokens to the builder thread
+int dyn_wait(sam_index* idx);                                          // until the builder thread has nothing left
+bool dyn_pop_ready(sam_index* idx, Delta* out);                        // next finished update, in order
+int dyn_full_image(sam_index* idx, Delta* out);                        // waits, drops queued updates, packs everything
+int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges);    // waits; states / transitions right now
+int dyn_refresh_csr(sam_index* idx);                                   // waits, refills the flat arrays for sam_export
+void dyn_counts(sam_index* idx, int64_t* queued, int64_t* built);      // tokens handed in / tokens indexed on the host
 }  // namespace samb200

@@ -1,0 +1,77 @@
+// Device side of the growing index (sm_100a). Included only by sam_capi.cu.
+//
+// Updates arrive in the staging area of the device blob as flat lists and are scattered into the
+// record array, the wide-edge array and the dense root table by the kernels below.  They run on the
+// caller's stream between decoding steps, so no walk ever sees a half-applied update.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "sam_index.h"
+
+namespace samb200 {
+
+// rec[ids[i]] = recs[i]; one thread per record, two 16-byte stores.
+__global__ void __launch_bounds__(256)
+scatter_records_kernel(StateRec* __restrict__ rec, const int32_t* __restrict__ ids,
+                       const StateRec* __restrict__ recs, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int4* src = reinterpret_cast<const int4*>(recs + i);
+    int4* dst = reinterpret_cast<int4*>(rec + ids[i]);
+    const int4 a = src[0], b = src[1];
+    dst[0] = a;
+    dst[1] = b;
+}
+
+struct SegDesc {
+    long long dst_off;   // first edge of the row in the wide array
+    int src_off;         // first edge of the row in the staged edge list
+    int len;
+};
+
+// One warp per rewritten wide row.
+__global__ void __launch_bounds__(256)
+copy_rows_kernel(Edge* __restrict__ wide, const SegDesc* __restrict__ segs, const Edge* __restrict__ staged, int n) {
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n) return;
+    const SegDesc g = segs[w];
+    const int2* src = reinterpret_cast<const int2*>(staged + g.src_off);
+    int2* dst = reinterpret_cast<int2*>(wide + g.dst_off);
+    for (int k = lane; k < g.len; k += 32) dst[k] = src[k];
+}
+
+// root_dst[tok[i]] = dst[i]
+__global__ void __launch_bounds__(256)
+scatter_root_kernel(int32_t* __restrict__ root_dst, const int32_t* __restrict__ tok, const int32_t* __restrict__ dst,
+                    int n, int span) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int t = tok[i];
+    if (t >= 0 && t < span) root_dst[t] = dst[i];
+}
+
+// After the text has grown, a stream's string of length L may belong to a state that was split off
+// its old one: the state of a string is the one with len(link(s)) < L <= len(s).  Climb suffix links
+// until that holds.  One thread per stream.
+__global__ void __launch_bounds__(128)
+renormalize_kernel(DeviceSam sam, int B, int* __restrict__ state, const int* __restrict__ matched_len) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int s = state[b];
+    const int L = matched_len[b];
+    if (s <= 0 || s >= sam.n_states || L < 0) return;      // the walk kernels reset such pairs themselves
+    const int s0 = s;
+    for (int hop = 0; hop < (1 << 30) && s != 0; ++hop) {
+        const int link = __ldg(&sam.rec[s].link);
+        if (link < 0 || link >= sam.n_states) break;
+        const int link_len = (link == 0) ? 0 : __ldg(&sam.rec[link].len);
+        if (L > link_len) break;
+        s = link;
+    }
+    if (s != s0) state[b] = s;
+}
+
+}  // namespace samb200

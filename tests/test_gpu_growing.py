@@ -1,0 +1,181 @@
+"""Parity of the growing index on the GPU with the oracle's growing automaton, tolerance 0.
+
+The text grows between decoding steps (new sessions, and the streams' own verified tokens); after
+every growth both sides renormalise the stream states, and every later output must still agree."""
+from __future__ import annotations
+
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2512_18337_b200 as S
+import workload as W
+from tests.cuda_backend import CudaBackend, bits_to_device
+from tests.oracle_backend import OracleBackend
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _i32(x):
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(DEV)
+
+
+def _hub_text(rng, n, sep):
+    body = rng.integers(0, 400, size=n).astype(np.int32)
+    body[::3] = rng.integers(0, 3, size=body[::3].shape[0])      # hubs: rows that keep growing
+    body[5::97] = sep
+    return body
+
+
+def _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm):
+    d = torch.full((B, K), -9, dtype=torch.int32, device=DEV)
+    nd = torch.full((B,), -9, dtype=torch.int32, device=DEV)
+    S.sam_draft(index.handle, B, st, ml, _i32(toks), toks.shape[1], _i32(n_new), K, mm, d, nd)
+    torch.cuda.synchronize()
+    d_o, nd_o = osam.draft_batch(st_o, ml_o, toks, n_new, K, mm)
+    assert (st.cpu().numpy() == st_o).all() and (ml.cpu().numpy() == ml_o).all()
+    assert (nd.cpu().numpy() == nd_o).all() and (d.cpu().numpy() == d_o).all()
+    return d_o, nd_o
+
+
+@pytest.mark.parametrize("seed,wide_per_token", [(0, None), (1, "0.8")])
+def test_draft_parity_while_the_text_grows(seed, wide_per_token, monkeypatch):
+    """With one wide edge of room per token (a tuning knob of the library) the wide rows run out of room
+    along the way and are laid out afresh (whole-image updates); the default keeps every update incremental."""
+    rng = np.random.default_rng(seed)
+    sep, K, mm, B, ld = 1000, 6, 2, 48, 12
+    text = _hub_text(rng, 3000, sep)
+    if wide_per_token is not None:
+        monkeypatch.setenv("SAM_B200_WIDE_EDGES_PER_TOKEN", wide_per_token)
+    index = S.SamIndex(text, [sep], max_tokens=12000, max_token_id=sep + 50)
+    osam = oracle.OracleSAM(text, [sep])
+    st = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ml = torch.zeros(B, dtype=torch.int32, device=DEV)
+    st_o = np.zeros(B, np.int32)
+    ml_o = np.zeros(B, np.int32)
+    hist = [[] for _ in range(B)]
+    moved = 0
+    for rnd in range(14):
+        toks = np.empty((B, ld), np.int32)
+        n_new = rng.integers(0, ld + 1, size=B).astype(np.int32)
+        for b in range(B):
+            start = int(rng.integers(0, osam.n - ld))
+            toks[b] = osam.corpus[start:start + ld]
+            noise = rng.random(ld) < 0.08
+            toks[b, noise] = rng.integers(0, sep + 40, size=int(noise.sum()))
+            hist[b] += [int(x) for x in toks[b, :n_new[b]]]
+        _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm)
+        # growth: a stream's own recent tokens as a new session, then fresh text with new token ids
+        b = int(rng.integers(0, B))
+        piece = np.concatenate([[sep], np.array(hist[b][-40:], np.int32), [sep],
+                                _hub_text(rng, int(rng.integers(50, 400)), sep),
+                                rng.integers(sep + 1, sep + 50, size=5).astype(np.int32)]).astype(np.int32)
+        osam.extend(piece)
+        S.sam_extend(index.handle, piece)
+        assert S.sam_sync(index.handle) == osam.n
+        before = st_o.copy()
+        osam.renormalize(st_o, ml_o)
+        moved += int((before != st_o).sum())
+        S.sam_renormalize(index.handle, B, st, ml)
+        torch.cuda.synchronize()
+        assert (st.cpu().numpy() == st_o).all()
+        # n_new = 0: the draft is re-emitted from the (moved) state over the grown text
+        _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, np.zeros(B, np.int32), K, mm)
+    assert moved > 0
+    inc, full, nbytes = S.sam_update_stats(index.handle)
+    assert inc + full == 14 and nbytes > 0
+    assert (full > 0) == (wide_per_token is not None)
+    ex, oe = S.sam_export(index.handle), osam.export()
+    for k in oe:
+        assert (ex[k] == oe[k]).all(), k
+
+
+def test_closed_loop_with_committed_tokens_appended():
+    """The fused step on a growing index: after every step the tokens some streams committed are appended
+    as new sessions, the device copy is synced, the states renormalised."""
+    cfg = W.CONFIGS[0].scaled(B=24, steps=12, sessions=6)
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    noise = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+    index = S.SamIndex(corpus, [cfg.separator], max_tokens=corpus.shape[0] + 4000, max_token_id=cfg.separator)
+    gpu = CudaBackend(cfg, corpus, bits_to_device(noise), index=index)
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    f_g, f_o = W.ClosedLoopFeeder(cfg, scripts, rowmax), W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = f_g.prime_tokens()
+    dg, ndg = gpu.prime(toks, n)
+    do, ndo = cpu.prime(toks, n)
+    assert (dg == do).all() and (ndg == ndo).all()
+    committed = [[] for _ in range(cfg.B)]
+    for t in range(cfg.steps):
+        outs = []
+        for be, f, (d, nd) in ((gpu, f_g, (dg, ndg)), (cpu, f_o, (do, ndo))):
+            ow = f.overwrites(t, d, nd)
+            keep = np.arange(ow["row"].shape[0])
+            saved = be.poke(ow["row"], ow["col"], ow["bits"], keep)
+            out = be.step(d, nd)
+            be.unpoke(ow["row"], ow["col"], saved)
+            f.advance(out["n_accepted"])
+            outs.append(out)
+        g, o = outs
+        for k in ("argmax", "accepted", "n_accepted", "state", "matched_len", "drafts", "n_draft"):
+            assert (g[k] == o[k]).all(), (t, k)
+        for b in range(cfg.B):
+            committed[b] += [int(x) for x in o["accepted"][b, :o["n_accepted"][b]]]
+        # every third step: two streams' output so far becomes part of the shared memory
+        if t % 3 == 2:
+            piece = []
+            for b in (t % cfg.B, (5 * t + 1) % cfg.B):
+                piece += [cfg.separator] + committed[b]
+            piece = np.array(piece, np.int32)
+            cpu.sam.extend(piece)
+            cpu.sam.renormalize(cpu.state, cpu.mlen)
+            S.sam_extend(index.handle, piece)
+            S.sam_sync(index.handle)
+            S.sam_renormalize(index.handle, cfg.B, gpu.state, gpu.mlen)
+            # the pending drafts came from the text before it grew; both sides re-emit them
+            z = np.zeros((cfg.B, 1), np.int32)
+            nz = np.zeros(cfg.B, np.int32)
+            dg, ndg = gpu.prime(z, nz)
+            do, ndo = cpu.prime(z, nz)
+            assert (dg == do).all() and (ndg == ndo).all()
+        else:
+            dg, ndg, do, ndo = g["drafts"], g["n_draft"], o["drafts"], o["n_draft"]
+
+
+def test_builder_thread_and_empty_start():
+    """An index that starts empty drafts nothing; text queued for the builder thread becomes visible only
+    after sam_sync; once everything is built and synced the drafts equal the oracle's."""
+    rng = np.random.default_rng(3)
+    sep, K, mm, B, ld = 500, 5, 2, 16, 10
+    index = S.SamIndex(np.zeros(0, np.int32), [sep], max_tokens=50000, max_token_id=sep)
+    text = _hub_text(rng, 20000, sep)
+    st = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ml = torch.zeros(B, dtype=torch.int32, device=DEV)
+    toks = np.stack([text[s:s + ld] for s in rng.integers(0, text.shape[0] - ld, size=B)]).astype(np.int32)
+    n_new = np.full(B, ld, np.int32)
+    d = torch.full((B, K), -9, dtype=torch.int32, device=DEV)
+    nd = torch.full((B,), -9, dtype=torch.int32, device=DEV)
+    S.sam_draft(index.handle, B, st, ml, _i32(toks), ld, _i32(n_new), K, mm, d, nd)
+    torch.cuda.synchronize()
+    assert int(nd.abs().sum()) == 0 and int(st.abs().sum()) == 0          # nothing indexed yet: no speculation
+    for piece in np.array_split(text, 23):
+        S.sam_extend(index.handle, piece, wait=False)
+    assert S.sam_pending(index.handle)[0] == text.shape[0]
+    assert S.sam_pending(index.handle)[2] == 0                            # the device has seen nothing so far
+    deadline = time.time() + 60
+    seen = 0
+    while seen < text.shape[0]:
+        seen = S.sam_sync(index.handle)                                   # whatever is finished so far
+        assert time.time() < deadline
+        time.sleep(0.002)
+    osam = oracle.OracleSAM(text, [sep])
+    st_o = np.zeros(B, np.int32)
+    ml_o = np.zeros(B, np.int32)
+    st.zero_(); ml.zero_()
+    _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm)
+    assert (ml_o == ld).all()

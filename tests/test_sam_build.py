@@ -95,3 +95,64 @@ def test_error_codes_without_a_device():
     with pytest.raises(S.SamError):
         S.sam_workspace_bytes(4, 33)
     assert "invalid" in S.sam_strerror(-1)
+
+
+# ------------------------------------------------------------------ growing index (host side)
+def _grow_and_compare(text, cuts, sep, wait_each=True):
+    parts = np.split(text, cuts)
+    h = S.sam_build_growing(parts[0], [sep], max_tokens=text.shape[0] + 5, max_token_id=int(max(text.max(), sep)))
+    try:
+        for p in parts[1:]:
+            S.sam_extend(h, p, wait=wait_each)
+        if not wait_each:
+            S.sam_extend(h, np.zeros(0, np.int32), wait=True)      # waits for the queue to drain
+        queued, built, on_dev = S.sam_pending(h)
+        assert queued == built == text.shape[0] and on_dev == 0
+        ex = S.sam_export(h)
+        S_, E_, nbytes = S.sam_sizes(h)
+    finally:
+        S.sam_free(h)
+    o = oracle.OracleSAM(text, [sep])
+    oe = o.export()
+    assert (S_, E_) == (o.n_states, o.n_edges)
+    for k in oe:
+        assert (ex[k] == oe[k]).all(), k
+    assert nbytes >= 32 * (2 * text.shape[0]) + 4 * text.shape[0]
+
+
+@pytest.mark.parametrize("sigma,n", [(1, 40), (2, 500), (3, 2000), (50, 3000)])
+def test_growing_index_equals_one_shot_build(sigma, n):
+    """Text that arrives in pieces (synchronously and through the builder thread's queue) yields the very
+    automaton, numbering included, that the oracle builds from the whole text."""
+    rng = np.random.default_rng(sigma * 1000 + n)
+    text = rng.integers(0, sigma, size=n).astype(np.int32)
+    cuts = np.sort(rng.choice(np.arange(1, n), size=min(7, n - 1), replace=False))
+    _grow_and_compare(text, cuts, sigma, wait_each=True)
+    _grow_and_compare(text, cuts, sigma, wait_each=False)
+
+
+def test_growing_index_from_empty_and_limits():
+    h = S.sam_build_growing(np.zeros(0, np.int32), [9], max_tokens=10, max_token_id=9)
+    try:
+        assert S.sam_sizes(h)[0] == 1                               # the root alone
+        S.sam_extend(h, np.array([1, 2, 1, 2, 9, 1], np.int32))
+        assert S.sam_pending(h)[:2] == (6, 6)
+        with pytest.raises(S.SamError) as e:
+            S.sam_extend(h, np.array([10], np.int32))               # id above max_token_id
+        assert e.value.status == -1
+        with pytest.raises(S.SamError) as e:
+            S.sam_extend(h, np.arange(5, dtype=np.int32))           # 6 + 5 > max_tokens
+        assert e.value.status == -6
+        ex = S.sam_export(h)
+        oe = oracle.OracleSAM(np.array([1, 2, 1, 2, 9, 1], np.int32), [9]).export()
+        for k in oe:
+            assert (ex[k] == oe[k]).all(), k
+    finally:
+        S.sam_free(h)
+    lib = S.binding._load()
+    hs = S.sam_build(np.array([1, 2, 3], np.int32), [9])
+    try:
+        assert lib.sam_extend(hs, None, 0) == -1                    # a one-shot index cannot grow
+        assert lib.sam_sync(hs, None, None) == -1
+    finally:
+        S.sam_free(hs)
