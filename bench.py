@@ -434,6 +434,94 @@ def run_reference(args):
     }))
 
 
+# ----------------------------------------------------------------------------- growing index
+def run_growing(args):
+    """Same closed loop on an index that keeps growing: every step the tokens all streams committed are
+    queued for the builder thread (one new session per step), and before each step whatever the thread has
+    finished is brought to the device (sam_sync) and the stream states are renormalised.  Prints its own JSON
+    line; the timed bracket of a step holds sync + renormalise + sam_step."""
+    import torch
+    import paper_2512_18337_b200 as S
+    from paper_2512_18337_b200.build import build
+    from tests.cuda_backend import CudaBackend
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    device = "cuda:0"
+    torch.cuda.set_device(device)
+    build()
+    base = W.CONFIGS[args.config]
+    cfg = base.scaled(steps=args.warmup + args.steps + 1)
+    corpus, logits, rowmax = make_inputs_gpu(cfg, device)
+    scripts = W.make_scripts(cfg, corpus)
+    room = (cfg.K + 2) * cfg.B * (args.warmup + args.steps + 2) + (1 << 20)
+    t0 = time.time()
+    index = S.SamIndex(corpus, [cfg.separator], device=device, max_tokens=cfg.n_corpus + room, max_token_id=cfg.separator)
+    t_build_upload = time.time() - t0
+    # builder throughput on its own: one large piece of fresh text, waited for
+    extra = W.make_corpus(cfg.scaled(sessions=max(1, (1 << 19) // cfg.session_len), seed=cfg.seed + 101))
+    t0 = time.time()
+    S.sam_extend(index.handle, extra)
+    t_extend = time.time() - t0
+    t0 = time.time()
+    S.sam_sync(index.handle)
+    torch.cuda.synchronize()
+    t_first_sync = time.time() - t0
+    stats0 = S.sam_update_stats(index.handle)
+
+    feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    be = CudaBackend(cfg, corpus, logits, index=index, device=device)
+    toks, n = feeder.prime_tokens()
+    drafts, n_draft = be.prime(toks, n)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    tokens = appended = 0
+    lag = []
+    for t in range(args.warmup + args.steps):
+        ow = feeder.overwrites(t, drafts, n_draft)
+        saved = be.poke(ow["row"], ow["col"], ow["bits"], np.arange(ow["row"].shape[0]))
+        i = t - args.warmup
+        if i >= 0:
+            torch.cuda._sleep(args.presleep_cycles)
+            ev[i][0].record()
+        S.sam_sync(index.handle)
+        S.sam_renormalize(index.handle, cfg.B, be.state, be.mlen)
+        be.launch_step()
+        if i >= 0:
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        n_acc = be.n_accepted.cpu().numpy()
+        acc = be.accepted.cpu().numpy()
+        drafts, n_draft = be.drafts.cpu().numpy(), be.n_draft.cpu().numpy()
+        be.unpoke(ow["row"], ow["col"], saved)
+        feeder.advance(n_acc)
+        piece = np.concatenate([[cfg.separator]] + [acc[b, :n_acc[b]] for b in range(cfg.B)]).astype(np.int32)
+        S.sam_extend(index.handle, piece, wait=False)
+        if i >= 0:
+            tokens += int(n_acc.sum())
+            appended += piece.shape[0]
+            q, bt, dv = S.sam_pending(index.handle)
+            lag.append(q - dv)
+    S.sam_extend(index.handle, np.zeros(0, np.int32))
+    S.sam_sync(index.handle)
+    torch.cuda.synchronize()
+    stats1 = S.sam_update_stats(index.handle)
+    ms = float(sum(a.elapsed_time(b) for a, b in ev))
+    print(json.dumps({
+        "metric": METRIC + "_growing_index", "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "dtype": "bf16 compare / int32", "data": "synthetic",
+        "config": {"workload": cfg.name + " + one appended session per step (all committed tokens)",
+                   "B": cfg.B, "K": cfg.K, "V": cfg.vocab, "timing": "CUDA events around sam_sync + sam_renormalize + sam_step"},
+        "appended_tokens_per_step": appended / args.steps,
+        "mean_tokens_not_yet_on_device_at_step_end": statistics.mean(lag),
+        "updates": {"incremental": stats1[0] - stats0[0], "full_images": stats1[1] - stats0[1],
+                    "h2d_bytes_per_step": (stats1[2] - stats0[2]) / args.steps},
+        "builder_thread_tokens_per_s": extra.shape[0] / t_extend,
+        "first_sync_s": t_first_sync, "first_sync_bytes": stats0[2], "build_and_upload_s": t_build_upload,
+        "device_bytes": index.device_bytes,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -451,10 +539,14 @@ def main():
                     help="steps run after the timed region with two kernels per step, to report each kernel's time")
     ap.add_argument("--cpu-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--growing", action="store_true",
+                    help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.growing:
+        run_growing(args)
     else:
         run_ours(args)
 
