@@ -32,6 +32,7 @@ struct Builder {
     std::vector<uint8_t> mark;                              // state already in `dirty`
     std::vector<int32_t> dirty;                             // non-root states to repack
     std::vector<std::pair<int32_t, int32_t>> root_changes;  // (token, destination) in order of change
+    std::vector<std::pair<int32_t, int32_t>> redirected;    // (state, token) of transitions that got a new destination
 
     void touch(int32_t s) {
         if (!track || s == 0) return;
@@ -41,6 +42,7 @@ struct Builder {
         for (int32_t s : dirty) mark[s] = 0;
         dirty.clear();
         root_changes.clear();
+        redirected.clear();
     }
 
     static uint64_t key_of(int32_t s, int32_t c) {
@@ -146,6 +148,7 @@ struct Builder {
                     e_dst[ex] = clone;
                     touch(p);
                     if (track && p == 0) root_changes.emplace_back(c, clone);
+                    if (track && p != 0) redirected.emplace_back(p, c);
                     p = link[p];
                 }
                 link[q] = clone;

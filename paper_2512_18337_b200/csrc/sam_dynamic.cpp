@@ -11,6 +11,7 @@
 // full image.
 #include <algorithm>
 #include <condition_variable>
+#include <climits>
 #include <cstdlib>
 #include <cstring>
 #include <deque>
@@ -30,6 +31,8 @@ struct DynIndex {
     std::vector<int32_t> corpus;
     int64_t max_tokens = 0, s_cap = 0, w_cap = 0, span_cap = 0;
     std::vector<int32_t> wide_off, wide_cap;   // per state: row offset / capacity in the device's wide array (-1 / 0: none)
+    std::vector<int32_t> packed_deg;           // per state: transitions its wide row held when it was last packed
+    std::vector<Edge> mirror;                  // host copy of the device's wide array (rows sorted by token)
     int64_t w_used = 0;
 
     std::thread worker;
@@ -50,36 +53,84 @@ int32_t pow2_at_least(int32_t d) {
     return c;
 }
 
-// Record of state s (not the root); a wide row is placed (or re-placed) when it outgrew its slot.
+// Record of state s (not the root).  A wide row lives, sorted, in the host mirror of the device's wide
+// array: a row that is new or has outgrown its slot is sorted and placed afresh; otherwise the
+// transitions added since the last packing (the newest nodes of the state's chain) are merged in and
+// redirected ones patched, so that a hub row with thousands of entries is never sorted again.
+// *first / *count tell which part of the row differs from what the device holds.
 // Returns false when the wide area is exhausted.
-bool pack_state(DynIndex& D, int32_t s, StateRec* r, std::vector<std::pair<int32_t, int32_t>>& row, bool* is_wide) {
+bool pack_state(DynIndex& D, int32_t s, StateRec* r, const std::pair<int32_t, int32_t>* redir, size_t n_redir,
+                std::vector<std::pair<int32_t, int32_t>>& tmp, int64_t* first, int64_t* count) {
     const Builder& b = D.b;
     r->len = b.len[s];
     r->link = b.link[s];
     r->firstpos = b.fpos[s];
     r->deg = b.deg[s];
     r->e[0] = r->e[1] = r->e[2] = r->e[3] = -1;
-    b.sorted_row(s, row);
+    *first = *count = 0;
     const int32_t d = b.deg[s];
-    *is_wide = d >= 3;
-    if (d >= 1 && d <= 2) {
-        r->e[0] = row[0].first;
-        r->e[1] = row[0].second;
-        if (d == 2) { r->e[2] = row[1].first; r->e[3] = row[1].second; }
-    } else if (d >= 3) {
-        if (static_cast<size_t>(s) >= D.wide_off.size()) {
-            D.wide_off.resize(b.len.size(), -1);
-            D.wide_cap.resize(b.len.size(), 0);
+    if (d <= 2) {
+        if (d >= 1) {
+            b.sorted_row(s, tmp);
+            r->e[0] = tmp[0].first;
+            r->e[1] = tmp[0].second;
+            if (d == 2) { r->e[2] = tmp[1].first; r->e[3] = tmp[1].second; }
         }
-        if (D.wide_cap[s] < d) {
-            const int32_t cap = pow2_at_least(d);
-            if (D.w_used + cap > D.w_cap) return false;
-            D.wide_off[s] = static_cast<int32_t>(D.w_used);
-            D.wide_cap[s] = cap;
-            D.w_used += cap;
-        }
-        r->e[0] = D.wide_off[s];
+        return true;
     }
+    if (static_cast<size_t>(s) >= D.wide_off.size()) {
+        D.wide_off.resize(b.len.size(), -1);
+        D.wide_cap.resize(b.len.size(), 0);
+        D.packed_deg.resize(b.len.size(), 0);
+    }
+    if (D.wide_cap[s] < d) {
+        // new slot, whole row
+        const int32_t cap = pow2_at_least(d);
+        if (D.w_used + cap > D.w_cap) return false;
+        D.wide_off[s] = static_cast<int32_t>(D.w_used);
+        D.wide_cap[s] = cap;
+        D.w_used += cap;
+        if (D.mirror.size() < static_cast<size_t>(D.w_used)) D.mirror.resize(static_cast<size_t>(D.w_used), Edge{-1, -1});
+        b.sorted_row(s, tmp);
+        Edge* row = D.mirror.data() + D.wide_off[s];
+        for (int32_t k = 0; k < d; ++k) row[k] = Edge{tmp[k].first, tmp[k].second};
+        *first = 0;
+        *count = d;
+    } else {
+        Edge* row = D.mirror.data() + D.wide_off[s];
+        const int32_t old = D.packed_deg[s];
+        int64_t lowest = d;                                   // lowest position written
+        const int32_t k_new = d - old;
+        if (k_new > 0) {
+            tmp.clear();
+            int32_t x = b.head[s];
+            for (int32_t k = 0; k < k_new; ++k, x = b.e_next[x]) tmp.emplace_back(b.e_tok[x], b.e_dst[x]);
+            std::sort(tmp.begin(), tmp.end());
+            int32_t i = old - 1, j = k_new - 1, w = d - 1;
+            while (j >= 0) {
+                if (i >= 0 && row[i].tok > tmp[j].first) row[w--] = row[i--];
+                else { row[w] = Edge{tmp[j].first, tmp[j].second}; --w; --j; }
+            }
+            lowest = w + 1;
+        }
+        for (size_t q = 0; q < n_redir; ++q) {
+            const int32_t tok = redir[q].second;
+            int32_t lo = 0, hi = d;
+            while (lo < hi) {
+                const int32_t mid = (lo + hi) >> 1;
+                if (row[mid].tok < tok) lo = mid + 1; else hi = mid;
+            }
+            if (lo < d && row[lo].tok == tok) {
+                const int32_t e = b.find(s, tok);
+                if (e >= 0) row[lo].dst = b.e_dst[e];
+                if (lo < lowest) lowest = lo;
+            }
+        }
+        *first = lowest;
+        *count = d - lowest;
+    }
+    D.packed_deg[s] = d;
+    r->e[0] = D.wide_off[s];
     return true;
 }
 
@@ -92,20 +143,15 @@ int pack_full(DynIndex& D, Delta* out) {
     out->all_root.assign(static_cast<size_t>(D.span_cap), -1);
     D.wide_off.assign(static_cast<size_t>(S), -1);
     D.wide_cap.assign(static_cast<size_t>(S), 0);
+    D.packed_deg.assign(static_cast<size_t>(S), 0);
+    D.mirror.clear();
     D.w_used = 0;
-    std::vector<std::pair<int32_t, int32_t>> row;
-    // first pass places the rows, second copies them (the total is known only after placing)
+    std::vector<std::pair<int32_t, int32_t>> tmp;
     for (int64_t s = 1; s < S; ++s) {
-        bool wide = false;
-        if (!pack_state(D, static_cast<int32_t>(s), &out->all_rec[s], row, &wide)) return SAM_ERR_TOO_LARGE;
+        int64_t first = 0, count = 0;
+        if (!pack_state(D, static_cast<int32_t>(s), &out->all_rec[s], nullptr, 0, tmp, &first, &count)) return SAM_ERR_TOO_LARGE;
     }
-    out->all_wide.assign(static_cast<size_t>(D.w_used), Edge{-1, -1});
-    for (int64_t s = 1; s < S; ++s) {
-        if (b.deg[s] < 3) continue;
-        b.sorted_row(static_cast<int32_t>(s), row);
-        Edge* dst = out->all_wide.data() + D.wide_off[s];
-        for (size_t k = 0; k < row.size(); ++k) dst[k] = Edge{row[k].first, row[k].second};
-    }
+    out->all_wide.assign(D.mirror.begin(), D.mirror.begin() + D.w_used);
     StateRec& r0 = out->all_rec[0];
     r0.len = 0; r0.link = -1; r0.firstpos = -1; r0.deg = b.deg[0];
     r0.e[0] = r0.e[1] = r0.e[2] = r0.e[3] = -1;
@@ -119,13 +165,16 @@ int pack_full(DynIndex& D, Delta* out) {
 // What the last chunk changed.
 int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
     Builder& b = D.b;
-    std::vector<std::pair<int32_t, int32_t>> row;
+    std::vector<std::pair<int32_t, int32_t>> tmp;
     out->rec_ids.reserve(b.dirty.size());
     out->recs.reserve(b.dirty.size());
+    std::sort(b.redirected.begin(), b.redirected.end());
     for (int32_t s : b.dirty) {
         StateRec r;
-        bool wide = false;
-        if (!pack_state(D, s, &r, row, &wide)) {
+        const auto lo = std::lower_bound(b.redirected.begin(), b.redirected.end(), std::make_pair(s, INT32_MIN));
+        const auto hi = std::lower_bound(lo, b.redirected.end(), std::make_pair(s + 1, INT32_MIN));
+        int64_t first = 0, count = 0;
+        if (!pack_state(D, s, &r, lo == hi ? nullptr : &*lo, static_cast<size_t>(hi - lo), tmp, &first, &count)) {
             // wide area exhausted: lay everything out afresh and send the whole image instead
             Delta fresh;
             const int rc = pack_full(D, &fresh);
@@ -134,13 +183,14 @@ int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
         }
         out->rec_ids.push_back(s);
         out->recs.push_back(r);
-        if (wide) {
+        if (count > 0) {
             WideSeg g;
-            g.dst_off = D.wide_off[s];
+            g.dst_off = D.wide_off[s] + first;
             g.src_off = static_cast<int64_t>(out->seg_edges.size());
-            g.len = static_cast<int32_t>(row.size());
+            g.len = static_cast<int32_t>(count);
             out->segs.push_back(g);
-            for (const auto& e : row) out->seg_edges.push_back(Edge{e.first, e.second});
+            const Edge* row = D.mirror.data() + D.wide_off[s] + first;
+            out->seg_edges.insert(out->seg_edges.end(), row, row + count);
         }
     }
     // root: the last change of a token wins
