@@ -75,6 +75,13 @@ def _load():
                                     _u16p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                     _i32p, _i32p, _i32p, _i32p, _i32p, _i32p, _i32p, C.c_int32,
                                     _i32p, _i32p, C.c_int32]
+        lib.oracle_step_ex.restype = None
+        lib.oracle_step_ex.argtypes = [C.c_void_p, _i32p, C.c_int64, _i32p, C.c_int32,
+                                       _u16p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                       _i32p, _i32p, _i32p, _i32p, _i32p, _i32p, _i32p, C.c_int32,
+                                       _i32p, _i32p, C.c_uint32, _i64p]
+        lib.oracle_speculation_enabled.restype = C.c_int32
+        lib.oracle_speculation_enabled.argtypes = [C.c_int64] * 4
         _lib = lib
     return _lib
 
@@ -182,9 +189,35 @@ class OracleSAM:
         return out
 
 
+NO_SPECULATION = 1
+SKIP_UNUSED_ROWS = 2
+
+
+def speculation_enabled(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:
+    return bool(_load().oracle_speculation_enabled(context_len, batch_size, max_context_len, max_batch_size))
+
+
 def argmax_row(row_bits: np.ndarray) -> int:
     r = np.ascontiguousarray(row_bits, dtype=np.uint16)
     return int(_load().oracle_argmax_row(_u16(r), r.shape[0]))
+
+
+def _step_ex(self, logits_bits, B, K, V, drafts, n_draft, state, matched_len, min_match, flags=0, counters=None):
+    """Step with options (NO_SPECULATION, SKIP_UNUSED_ROWS) and running counters (int64[6], updated in place)."""
+    lg = logits_bits.reshape(B * (K + 1), -1)
+    out = dict(argmax=np.empty((B, K + 1), np.int32), accepted=np.empty((B, K + 1), np.int32),
+               n_accepted=np.empty(B, np.int32), drafts=np.empty((B, K), np.int32),
+               n_draft=np.empty(B, np.int32))
+    cp = counters.ctypes.data_as(_i64p) if counters is not None else None
+    self.lib.oracle_step_ex(self.h, _i32(self.corpus), self.n, _i32(self.seps), self.seps.shape[0],
+                            _u16(lg), lg.shape[1], B, K, V, _i32(drafts), _i32(n_draft),
+                            _i32(out["argmax"]), _i32(out["accepted"]), _i32(out["n_accepted"]),
+                            _i32(state), _i32(matched_len), min_match,
+                            _i32(out["drafts"]), _i32(out["n_draft"]), flags, cp)
+    return out
+
+
+OracleSAM.step_ex = _step_ex
 
 
 def argmax_batch(logits_bits: np.ndarray, V: int | None = None, threads: int = 1) -> np.ndarray:

@@ -356,3 +356,67 @@ void oracle_step(const osam *a, const int32_t *corpus, int64_t n,
                        accepted, K + 1, n_accepted, K, min_match,
                        next_drafts, next_n_draft, threads);
 }
+
+/* ---- step with options and running statistics ------------------------------ */
+/* Options of a step:
+ *   ORACLE_NO_SPECULATION (Section 5.4.3 "Adaptive switch", Algorithm 3 step 4): speculation is off
+ *     for this step - every stream verifies an empty proposal (plain decoding: one row, one committed
+ *     token), the automaton walk still follows the committed token, and no new draft is emitted.
+ *   ORACLE_SKIP_UNUSED_ROWS: only rows 0..n_draft[b] of stream b are looked at (row n_draft[b] gives
+ *     the model's own token after a full accept); the rows beyond get index -1.
+ * Statistics (Section 6.5): OTE = committed tokens / verification passes; SHR = accepted speculative
+ * tokens / proposed speculative tokens over the steps with a non-empty proposal.
+ * counters[0..5] += { passes, committed tokens, proposed draft tokens, accepted draft tokens,
+ *                     non-empty proposals, rows looked at }. */
+#define ORACLE_NO_SPECULATION   1
+#define ORACLE_SKIP_UNUSED_ROWS 2
+
+void oracle_step_ex(const osam *a, const int32_t *corpus, int64_t n,
+                    const int32_t *seps, int32_t n_sep,
+                    const uint16_t *logits, int64_t row_stride, int32_t B, int32_t K, int32_t V,
+                    const int32_t *drafts, const int32_t *n_draft,
+                    int32_t *argmax_out, int32_t *accepted, int32_t *n_accepted,
+                    int32_t *state, int32_t *matched_len, int32_t min_match,
+                    int32_t *next_drafts, int32_t *next_n_draft,
+                    uint32_t flags, int64_t *counters)
+{
+    for (int32_t b = 0; b < B; b++) {
+        int32_t nd = n_draft[b];
+        if (nd < 0) nd = 0;
+        if (nd > K) nd = K;
+        if (flags & ORACLE_NO_SPECULATION) nd = 0;
+        int32_t *am = argmax_out + (int64_t)b * (K + 1);
+        int64_t rows = 0;
+        for (int32_t j = 0; j <= K; j++) {
+            if ((flags & ORACLE_SKIP_UNUSED_ROWS) && j > nd) { am[j] = -1; continue; }
+            am[j] = oracle_argmax_row(logits + ((int64_t)b * (K + 1) + j) * row_stride, V);
+            rows++;
+        }
+        int32_t *acc = accepted + (int64_t)b * (K + 1);
+        n_accepted[b] = oracle_accept(drafts + (int64_t)b * K, nd, am, K, acc);
+        oracle_walk(a, &state[b], &matched_len[b], acc, n_accepted[b]);
+        int32_t *nx = next_drafts + (int64_t)b * K;
+        if (flags & ORACLE_NO_SPECULATION) {
+            for (int32_t j = 0; j < K; j++) nx[j] = -1;
+            next_n_draft[b] = 0;
+        } else {
+            next_n_draft[b] = oracle_draft(a, corpus, n, seps, n_sep, state[b], matched_len[b], K, min_match, nx);
+        }
+        if (counters) {
+            counters[0] += 1;
+            counters[1] += n_accepted[b];
+            counters[2] += nd;
+            counters[3] += n_accepted[b] - 1;
+            counters[4] += nd > 0;
+            counters[5] += rows;
+        }
+    }
+}
+
+/* The adaptive switch (Section 5.4.3; Algorithm 3 step 4): speculation stays on unless the context
+ * length or the batch size exceeds its threshold. */
+int32_t oracle_speculation_enabled(int64_t context_len, int64_t batch_size,
+                                   int64_t max_context_len, int64_t max_batch_size)
+{
+    return !(context_len > max_context_len || batch_size > max_batch_size);
+}
