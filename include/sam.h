@@ -88,7 +88,7 @@ void sam_free(sam_index* idx);
 
 /* Bytes of device scratch sam_verify / sam_step need for B streams and draft length K
  * (one 64-bit partial result per logits row, the walk-ahead states of every draft position, one
- * completion counter per stream and a status word).  Returns a negative SAM_ERR_* on bad sizes. */
+ * completion counter per stream, a row list and a status word).  Returns a negative SAM_ERR_* on bad sizes. */
 int64_t sam_workspace_bytes(int32_t B, int32_t K);
 
 /* Zero-fills the scratch (device, 8-byte aligned) on the stream.  Required once before the
@@ -158,6 +158,44 @@ int sam_step(const sam_index* idx,
              int32_t* state, int32_t* matched_len, int32_t min_match,
              int32_t* next_drafts, int32_t* next_n_draft,
              void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* Step options and running statistics.
+ *   SAM_STEP_NO_SPECULATION   (Section 5.4.3 "Adaptive switch"; Algorithm 3 step 4) speculation is off
+ *       for this call: every stream verifies an empty proposal (plain decoding: row 0 gives the one
+ *       committed token), the automaton still follows that token so that drafting can resume at once,
+ *       and no new draft is emitted (next_n_draft = 0, next_drafts = -1).
+ *   SAM_STEP_SKIP_UNUSED_ROWS only rows 0..n_draft[b] of stream b are read (row n_draft[b] supplies the
+ *       model's own token after a full accept); argmax_out of the rows beyond is -1.  A small kernel
+ *       lists the used rows first, then the argmax kernel streams only those - the bytes read per call
+ *       drop from B*(K+1) rows to sum(n_draft)+B rows.
+ *   counters  device, int64[SAM_N_COUNTERS], 8-byte aligned, or NULL.  Every call ADDS, per stream:
+ *       [0] verification passes (1), [1] committed tokens, [2] proposed draft tokens, [3] accepted draft
+ *       tokens, [4] non-empty proposals, [5] logits rows read.  Section 6.5: OTE = [1]/[0],
+ *       SHR = [3]/[2] (or [3]/(K*[4]) when every proposal counts as K tokens).  The caller zeroes and
+ *       reads them (a device-to-host copy of 48 bytes whenever it wants the figures).
+ * Everything else is as in sam_verify / sam_step, which are these calls with flags = 0, counters = NULL. */
+#define SAM_STEP_NO_SPECULATION   1u
+#define SAM_STEP_SKIP_UNUSED_ROWS 2u
+#define SAM_N_COUNTERS            6
+int sam_verify_ex(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                  const int32_t* drafts, const int32_t* n_draft,
+                  int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                  uint32_t flags, int64_t* counters,
+                  void* workspace, int64_t workspace_bytes, void* cuda_stream);
+int sam_step_ex(const sam_index* idx,
+                const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                const int32_t* drafts, const int32_t* n_draft,
+                int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                int32_t* state, int32_t* matched_len, int32_t min_match,
+                int32_t* next_drafts, int32_t* next_n_draft,
+                uint32_t flags, int64_t* counters,
+                void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* The adaptive switch itself (Section 5.4.3; Algorithm 3 step 4): 1 = keep speculating, 0 = fall back
+ * to plain decoding because the context length or the batch size exceeds its threshold.  The
+ * thresholds are deployment-specific ("empirically determined" in the paper); a host-side helper,
+ * no device work. */
+int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_context_len, int64_t max_batch_size);
 
 /* Allocation-free form of sam_verify (a packaging variant; the paper has no counterpart).
  * Some callers cannot obtain device scratch at all: a plugin running inside a serving engine

@@ -37,6 +37,10 @@ _SIGNATURES = {
     "sam_verify": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
     "sam_step": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                            _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_verify_ex": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, C.c_uint32, _vp, _vp, _i64, _vp]),
+    "sam_step_ex": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                              _vp, _vp, _i32, _vp, _vp, C.c_uint32, _vp, _vp, _i64, _vp]),
+    "sam_adaptive_switch": (C.c_int, [_i64, _i64, _i64, _i64]),
     "sam_verify_static": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
@@ -250,6 +254,33 @@ def sam_step(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, a
                             _dev(argmax_out), _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len),
                             min_match, _dev(next_drafts), _dev(next_n_draft), _dev(workspace), workspace_bytes,
                             _stream(stream)), "sam_step")
+
+
+SAM_STEP_NO_SPECULATION = 1
+SAM_STEP_SKIP_UNUSED_ROWS = 2
+SAM_N_COUNTERS = 6
+
+
+def sam_verify_ex(logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                  flags, counters, workspace, workspace_bytes, stream=None):
+    """sam_verify with step options (SAM_STEP_*) and optional device counters (int64[SAM_N_COUNTERS])."""
+    _check(_load().sam_verify_ex(_dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft), _dev(argmax_out),
+                                 _dev(accepted), _dev(n_accepted), flags, _dev(counters), _dev(workspace),
+                                 workspace_bytes, _stream(stream)), "sam_verify_ex")
+
+
+def sam_step_ex(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                state, matched_len, min_match, next_drafts, next_n_draft, flags, counters,
+                workspace, workspace_bytes, stream=None):
+    """sam_step with step options (SAM_STEP_*) and optional device counters (int64[SAM_N_COUNTERS])."""
+    _check(_load().sam_step_ex(handle, _dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft),
+                               _dev(argmax_out), _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len),
+                               min_match, _dev(next_drafts), _dev(next_n_draft), flags, _dev(counters),
+                               _dev(workspace), workspace_bytes, _stream(stream)), "sam_step_ex")
+
+
+def sam_adaptive_switch(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:
+    return bool(_load().sam_adaptive_switch(context_len, batch_size, max_context_len, max_batch_size))
 
 
 def _hostptr(a) -> Optional[int]:

@@ -179,7 +179,8 @@ __global__ void __launch_bounds__(kBulkThreads, 1)
 argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
                    int tiles_per_row, int tile_vec, unsigned long long* __restrict__ keys,
                    int* __restrict__ status, const __grid_constant__ DeviceSam sam,
-                   const __grid_constant__ PreWalk pw, const __grid_constant__ FusedTail ft) {
+                   const __grid_constant__ PreWalk pw, const __grid_constant__ FusedTail ft,
+                   const __grid_constant__ RowMap rm) {
     // tile_vec <= kBulkTileVec: vectors per tile, chosen by the host so that a row splits into
     // tiles_per_row nearly equal tiles (large tiles amortise the per-tile hand-shake best).
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -190,11 +191,13 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const long long total = R * tiles_per_row;
+    // with a row list the number of rows is only known on the device, and a CTA's share may be empty
+    const long long n_all = (rm.list != nullptr) ? __ldg(rm.n_rows) : R;
+    const long long total = n_all * tiles_per_row;
     const long long t0 = total * blockIdx.x / gridDim.x;
-    const long long t1 = total * (blockIdx.x + 1) / gridDim.x;      // t1 > t0: the grid never exceeds the tile count
-    const long long row_first = t0 / tiles_per_row;
-    const int n_rows = static_cast<int>((t1 - 1) / tiles_per_row - row_first + 1);   // rows this CTA touches
+    const long long t1 = total * (blockIdx.x + 1) / gridDim.x;
+    const long long row_first = t0 / tiles_per_row;      // position in the list (or the row itself without one)
+    const int n_rows = (t1 > t0) ? static_cast<int>((t1 - 1) / tiles_per_row - row_first + 1) : 0;   // rows this CTA touches
     const int nvec_row = V >> 3;               // whole 16-byte vectors per row (rows are 16-byte aligned)
     const int ragged = V & 7;                  // trailing elements read with plain loads
 
@@ -229,6 +232,8 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             uint32_t use = 0;
             const uint64_t policy = l2_evict_first_policy();
             for (long long t = t0; t < t1; ++t, ++it) {
+                // with a row list the row number is fetched before the wait, off the path of the copy
+                const long long arow = (rm.list != nullptr) ? __ldg(rm.list + row) : row;
                 if (!mbar_wait_bounded(&sh->empty[s], (use & 1u) ^ 1u, abort)) { ok = false; break; }
                 const int v0 = tile * tile_vec;
                 const int nv = max(0, min(tile_vec, nvec_row - v0));
@@ -236,7 +241,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                     const uint32_t bytes = static_cast<uint32_t>(nv) * 16u;
                     mbar_arrive_expect_tx(&sh->full[s], bytes);
                     bulk_load(stage_base + static_cast<size_t>(s) * kBulkTileBytes,
-                              reinterpret_cast<const uint4*>(logits + row * stride) + v0, bytes, &sh->full[s], policy);
+                              reinterpret_cast<const uint4*>(logits + arow * stride) + v0, bytes, &sh->full[s], policy);
                 } else {
                     mbar_arrive(&sh->full[s]);      // nothing to copy (row shorter than one vector)
                 }
@@ -275,7 +280,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             const int n = min(32, p - done_rows);
             if (lane < n) {
                 const int i = done_rows + lane;
-                const long long row = row_first + i;
+                const long long row = (rm.list != nullptr) ? __ldg(rm.list + row_first + i) : row_first + i;
                 const unsigned long long* c = cand + static_cast<size_t>(i % kRowSlots) * kBulkConsumerWarps;
                 unsigned long long k = 0ull;
 #pragma unroll
@@ -343,7 +348,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         // Hands the finished row over to the finisher: candidate into the row's slot, then the progress counter.
         auto flush = [&]() -> bool {
             if (cur_row < 0) return true;
-            unsigned long long k = (best_idx >= 0) ? pack_candidate(best, static_cast<unsigned>(best_idx)) : 0ull;
+            unsigned long long k = (best_idx >= 0) ? pack_candidate(best, static_cast<unsigned>(best_idx + rm.v_offset)) : 0ull;
             if (first_nan) k = kCandidateFirstIsNaN;
             k = warp_max_u64(k);
             int good = 1;
@@ -386,7 +391,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                 const int q = ct + i * kBulkConsumers;
                 if (q < nv) {
                     const uint4 v = st[q];
-                    if (i == 0 && ct == 0 && tile == 0) first_nan = bf16_bits_nan(v.x & 0xFFFFu);
+                    if (i == 0 && ct == 0 && tile == 0) first_nan = rm.v_offset == 0 && bf16_bits_nan(v.x & 0xFFFFu);
                     const float m = vec_max(v);
                     if (m > best) { best = m; bestq = q; }
                 }
@@ -399,9 +404,10 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             if (lane == 0) mbar_arrive(&sh->empty[s]);
             if (ragged != 0 && tile == tiles_per_row - 1 && ct < ragged) {
                 const int e = nvec_row * 8 + ct;
-                const unsigned short b = __ldg(reinterpret_cast<const unsigned short*>(logits + row * stride) + e);
+                const long long arow = (rm.list != nullptr) ? __ldg(rm.list + row) : row;
+                const unsigned short b = __ldg(reinterpret_cast<const unsigned short*>(logits + arow * stride) + e);
                 const float x = __uint_as_float(static_cast<unsigned>(b) << 16);
-                if (e == 0) first_nan = bf16_bits_nan(b);         // rows shorter than one vector
+                if (e == 0) first_nan = rm.v_offset == 0 && bf16_bits_nan(b);   // rows shorter than one vector
                 if (x > best) { best = x; best_idx = e; }
             }
             if (++tile == tiles_per_row) { tile = 0; ++row; }

@@ -87,13 +87,16 @@ inline int* status_word(unsigned long long* keys, int64_t R) {
 
 // Partial results land in keys[R]; `status` receives a non-zero code if a kernel gives up on an
 // internal wait.
-// Layout of the verification scratch: keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B]
+// Layout of the verification scratch:
+// keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B] | row_list[R] | n_rows (256 B)
 struct Scratch {
     unsigned long long* keys;
     int* status;
     int* pre_state;
     int* pre_len;
     int* done;
+    int* row_list;
+    int* n_rows;
     int64_t bytes;
 };
 Scratch scratch_layout(void* base, int32_t B, int32_t K) {
@@ -107,6 +110,8 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K) {
     s.pre_state = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * K * 4);
     s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * K * 4);
     s.done = reinterpret_cast<int*>(p + o);                 o = up(o + static_cast<int64_t>(B) * 4);
+    s.row_list = reinterpret_cast<int*>(p + o);             o = up(o + R * 4);
+    s.n_rows = reinterpret_cast<int*>(p + o);               o += 256;
     s.bytes = o;
     return s;
 }
@@ -118,13 +123,14 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K) {
 int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
                   int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
                   bool* did_prewalk = nullptr, const AcceptArgs* tail = nullptr, int tail_mode = 0,
-                  int* done = nullptr, bool* did_tail = nullptr) {
+                  int* done = nullptr, bool* did_tail = nullptr, const RowMap* rmap = nullptr) {
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != SAM_OK) return rc;
     const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0;
     const bool bulk = rows_aligned && g_argmax_variant != 1;
+    const RowMap rm = rmap ? *rmap : RowMap{nullptr, nullptr, 0};
     if (did_prewalk) *did_prewalk = false;
     if (did_tail) *did_tail = false;
     if (bulk) {
@@ -145,7 +151,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid < 1) grid = 1;
         const bool prewalk = pw != nullptr && pw->enabled != 0;
         FusedTail ft{};
-        if (tail != nullptr && done != nullptr && g_argmax_variant == 2) {
+        if (tail != nullptr && done != nullptr && g_argmax_variant == 2 && rm.list == nullptr) {
             // a CTA can be handed at most the streams that overlap its contiguous range of rows
             const int64_t rows_per_cta = (total + grid - 1) / grid / tiles_per_row + 2;
             const int64_t streams_per_cta = rows_per_cta / (tail->K + 1) + 2;
@@ -159,7 +165,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         }
         argmax_bulk_kernel<<<static_cast<unsigned>(grid), kBulkThreads, kBulkSmemBytes, st>>>(
             static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status,
-            sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{}, ft);
+            sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{}, ft, rm);
         ++g_launches;
         if (did_prewalk) *did_prewalk = prewalk;
         if (did_tail) *did_tail = ft.mode != 0;
@@ -171,7 +177,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid > total) grid = total;
         if (grid < 1) grid = 1;
         argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys);
+            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, keys, rm);
         ++g_launches;
     }
     SAM_CUDA(cudaGetLastError());
@@ -452,10 +458,13 @@ int sam_draft(const sam_index* idx, int32_t B, int32_t* state, int32_t* matched_
     return SAM_OK;
 }
 
-int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
-               const int32_t* drafts, const int32_t* n_draft,
-               int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
-               void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+int sam_verify_ex(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                  const int32_t* drafts, const int32_t* n_draft,
+                  int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                  uint32_t flags, int64_t* counters,
+                  void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    if (flags & ~static_cast<uint32_t>(SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS)) return SAM_ERR_INVALID_ARG;
+    if (counters && !aligned(counters, 8)) return SAM_ERR_INVALID_ARG;
     int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
                                n_accepted, workspace, workspace_bytes);
     if (rc != SAM_OK || B == 0) return rc;
@@ -464,13 +473,75 @@ int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int
     const Scratch sc = scratch_layout(workspace, B, K);
     const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
                         argmax_out, accepted, n_accepted, sc.keys, nullptr, nullptr, 1, nullptr, nullptr,
-                        nullptr, nullptr};
+                        nullptr, nullptr, flags, reinterpret_cast<unsigned long long*>(counters)};
+    RowMap rm{nullptr, nullptr, 0};
+    if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
+        build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.n_rows);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+        rm.list = sc.row_list;
+        rm.n_rows = sc.n_rows;
+    }
     bool did_tail = false;
     rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, nullptr, nullptr, nullptr,
-                       &aa, kTailVerifyOnly, sc.done, &did_tail);
+                       &aa, kTailVerifyOnly, sc.done, &did_tail, &rm);
     if (rc != SAM_OK) return rc;
     if (!did_tail) {
         rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
+        if (rc != SAM_OK) return rc;
+    }
+    prof_mark(2, st);
+    prof_done();
+    return SAM_OK;
+}
+
+int sam_verify(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+               const int32_t* drafts, const int32_t* n_draft,
+               int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+               void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    return sam_verify_ex(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                         0, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+int sam_step_ex(const sam_index* idx,
+                const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                const int32_t* drafts, const int32_t* n_draft,
+                int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                int32_t* state, int32_t* matched_len, int32_t min_match,
+                int32_t* next_drafts, int32_t* next_n_draft,
+                uint32_t flags, int64_t* counters,
+                void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    if (!idx || min_match < 1) return SAM_ERR_INVALID_ARG;
+    if (flags & ~static_cast<uint32_t>(SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS)) return SAM_ERR_INVALID_ARG;
+    if (counters && !aligned(counters, 8)) return SAM_ERR_INVALID_ARG;
+    int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
+                               n_accepted, workspace, workspace_bytes);
+    if (rc != SAM_OK) return rc;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!state || !matched_len || !next_drafts || !next_n_draft) return SAM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    const Scratch sc = scratch_layout(workspace, B, K);
+    PreWalk pw{state, matched_len, drafts, n_draft, sc.pre_state, sc.pre_len, B, K, 1,
+               (flags & SAM_STEP_NO_SPECULATION) ? 1 : 0};
+    AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                  argmax_out, accepted, n_accepted, sc.keys, state, matched_len, min_match, next_drafts,
+                  next_n_draft, sc.pre_state, sc.pre_len, flags, reinterpret_cast<unsigned long long*>(counters)};
+    RowMap rm{nullptr, nullptr, 0};
+    if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
+        build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.n_rows);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+        rm.list = sc.row_list;
+        rm.n_rows = sc.n_rows;
+    }
+    bool did_prewalk = false, did_tail = false;
+    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, &idx->dev, &pw, &did_prewalk,
+                       &aa, kTailResume, sc.done, &did_tail, &rm);
+    if (rc != SAM_OK) return rc;
+    if (!did_tail) {
+        rc = did_prewalk ? launch_accept<kTailResume>(idx->dev, aa, st) : launch_accept<kTailFullWalk>(idx->dev, aa, st);
         if (rc != SAM_OK) return rc;
     }
     prof_mark(2, st);
@@ -485,31 +556,13 @@ int sam_step(const sam_index* idx,
              int32_t* state, int32_t* matched_len, int32_t min_match,
              int32_t* next_drafts, int32_t* next_n_draft,
              void* workspace, int64_t workspace_bytes, void* cuda_stream) {
-    if (!idx || min_match < 1) return SAM_ERR_INVALID_ARG;
-    int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
-                               n_accepted, workspace, workspace_bytes);
-    if (rc != SAM_OK) return rc;
-    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
-    if (B == 0) return SAM_OK;
-    if (!state || !matched_len || !next_drafts || !next_n_draft) return SAM_ERR_INVALID_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const int64_t R = static_cast<int64_t>(B) * (K + 1);
-    const Scratch sc = scratch_layout(workspace, B, K);
-    PreWalk pw{state, matched_len, drafts, n_draft, sc.pre_state, sc.pre_len, B, K, 1};
-    AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
-                  argmax_out, accepted, n_accepted, sc.keys, state, matched_len, min_match, next_drafts,
-                  next_n_draft, sc.pre_state, sc.pre_len};
-    bool did_prewalk = false, did_tail = false;
-    rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, &idx->dev, &pw, &did_prewalk,
-                       &aa, kTailResume, sc.done, &did_tail);
-    if (rc != SAM_OK) return rc;
-    if (!did_tail) {
-        rc = did_prewalk ? launch_accept<kTailResume>(idx->dev, aa, st) : launch_accept<kTailFullWalk>(idx->dev, aa, st);
-        if (rc != SAM_OK) return rc;
-    }
-    prof_mark(2, st);
-    prof_done();
-    return SAM_OK;
+    return sam_step_ex(idx, logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                       state, matched_len, min_match, next_drafts, next_n_draft, 0, nullptr,
+                       workspace, workspace_bytes, cuda_stream);
+}
+
+int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_context_len, int64_t max_batch_size) {
+    return (context_len > max_context_len || batch_size > max_batch_size) ? 0 : 1;
 }
 
 namespace {
@@ -585,7 +638,7 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     if (rc != SAM_OK) return rc;
     const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
                         argmax_out, accepted, n_accepted, keys, nullptr, nullptr, 1, nullptr, nullptr,
-                        nullptr, nullptr};
+                        nullptr, nullptr, 0u, nullptr};
     rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
     if (rc != SAM_OK) return rc;
     prof_mark(2, st);

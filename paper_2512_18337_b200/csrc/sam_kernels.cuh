@@ -177,13 +177,14 @@ struct PreWalk {
     int* pre_len;            // [B, K] matched_len after drafts[b, 0..j]
     int B, K;
     int enabled;
+    int no_spec;             // speculation is off for this step: every proposal counts as empty
 };
 
 __device__ __forceinline__ void prewalk_stream(const DeviceSam& sam, const PreWalk& pw, int b, int lane) {
     int s = pw.state[b];
     int L = pw.matched_len[b];
     sanitize_stream_state(sam, s, L);
-    const int nd = max(0, min(pw.n_draft[b], pw.K));
+    const int nd = pw.no_spec ? 0 : max(0, min(pw.n_draft[b], pw.K));
     const int d = (lane < nd) ? pw.drafts[static_cast<long long>(b) * pw.K + lane] : -1;
     if (nd == 0) return;
     RecRegs r = (s == 0) ? root_rec() : load_rec(sam, s);
@@ -289,18 +290,65 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+// Optional indirection and offset for the argmax kernels.
+//   list / n_rows: only the rows list[0..*n_rows) are reduced, in that order (both in device memory);
+//                  nullptr: all rows 0..R-1.
+//   v_offset:      added to every index (the logits are columns v_offset.. of a wider vocabulary).
+struct RowMap {
+    const int* list;
+    const int* n_rows;
+    int v_offset;
+};
+
+// Step options (same values as SAM_STEP_* in sam.h).
+constexpr unsigned kNoSpeculation = 1u, kSkipUnusedRows = 2u;
+
+// Rows 0..n_draft[b] of every stream, in stream order (n_draft clamped to 0..K, or 0 when speculation
+// is off); one CTA, a block-wide running sum.  *n_rows receives the count.
+__global__ void __launch_bounds__(1024)
+build_row_list_kernel(const int* __restrict__ n_draft, int B, int K, unsigned flags,
+                      int* __restrict__ list, int* __restrict__ n_rows) {
+    __shared__ int warp_sum[32];
+    __shared__ int carry;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < B; base += blockDim.x) {
+        const int b = base + threadIdx.x;
+        int need = 0;
+        if (b < B) need = ((flags & kNoSpeculation) ? 0 : max(0, min(n_draft[b], K))) + 1;
+        int incl = need;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += o;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        int before = carry;
+        for (int w = 0; w < warp; ++w) before += warp_sum[w];
+        const int start = before + incl - need;
+        for (int j = 0; j < need; ++j) list[start + j] = b * (K + 1) + j;
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry = before + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *n_rows = carry;
+}
+
 constexpr int kArgmaxThreads = 256;
 constexpr int kTileVec = 1024;    // 16-byte vectors per tile: 16 KB
 constexpr int kVecPerThread = kTileVec / kArgmaxThreads;
 
 // Turn a thread's (best value, vector index) into a packed candidate by re-reading that one
 // vector (an L2 hit: it was streamed moments ago) and locating the first equal element.
-__device__ __forceinline__ unsigned long long resolve_candidate(const RowView& rv, int V, float best, int bestq) {
+__device__ __forceinline__ unsigned long long resolve_candidate(const RowView& rv, int V, float best, int bestq,
+                                                                int v_offset) {
     if (bestq < 0) return 0ull;
     uint4 v = __ldg(rv.vec + bestq);
     if (bestq == 0 || bestq == rv.nvec - 1) mask_vector(v, bestq, rv.off, V);
     const int e = first_equal(v, best);
-    const unsigned idx = static_cast<unsigned>(bestq * 8 + e - rv.off);
+    const unsigned idx = static_cast<unsigned>(bestq * 8 + e - rv.off + v_offset);
     return pack_candidate(best, idx);
 }
 
@@ -318,7 +366,8 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
 // results of a row meet in keys[row] through a 64-bit atomic max.
 __global__ void __launch_bounds__(kArgmaxThreads)
 argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
-                     int tiles_per_row, unsigned long long* __restrict__ keys) {
+                     int tiles_per_row, unsigned long long* __restrict__ keys, RowMap rm) {
+    if (rm.list != nullptr) R = __ldg(rm.n_rows);
     const long long total = R * tiles_per_row;
     const long long t0 = total * blockIdx.x / gridDim.x;
     const long long t1 = total * (blockIdx.x + 1) / gridDim.x;
@@ -331,14 +380,15 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
 
     auto flush = [&]() {
         if (cur_row < 0) return;
-        unsigned long long k = first_nan ? kCandidateFirstIsNaN : resolve_candidate(rv, V, best, bestq);
+        unsigned long long k = first_nan ? kCandidateFirstIsNaN : resolve_candidate(rv, V, best, bestq, rm.v_offset);
         k = warp_max_u64(k);
         if (lane == 0 && k != 0ull) atomicMax(keys + cur_row, k);
     };
 
     for (long long t = t0; t < t1; ++t) {
-        const long long row = t / tiles_per_row;
-        const int tile = static_cast<int>(t - row * tiles_per_row);
+        const long long vrow = t / tiles_per_row;
+        const int tile = static_cast<int>(t - vrow * tiles_per_row);
+        const long long row = (rm.list != nullptr) ? __ldg(rm.list + vrow) : vrow;
         if (row != cur_row) {
             flush();
             cur_row = row;
@@ -362,7 +412,7 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
                 if (q == 0) {
                     const int h = rv.off >> 1;
                     const unsigned pair = (h == 0) ? v[i].x : (h == 1) ? v[i].y : (h == 2) ? v[i].z : v[i].w;
-                    first_nan = bf16_bits_nan((rv.off & 1) ? (pair >> 16) : (pair & 0xFFFFu));
+                    first_nan = rm.v_offset == 0 && bf16_bits_nan((rv.off & 1) ? (pair >> 16) : (pair & 0xFFFFu));
                 }
                 if (q == 0 || q == rv.nvec - 1) mask_vector(v[i], q, rv.off, V);
                 const float m = vec_max(v[i]);
@@ -398,6 +448,8 @@ struct AcceptArgs {
     int* next_n_draft;        // [B]
     const int* pre_state;     // [B, K] walk-ahead results (kTailResume)
     const int* pre_len;       // [B, K]
+    unsigned flags;           // kNoSpeculation | kSkipUnusedRows
+    unsigned long long* counters;   // [6] running statistics, or nullptr
 };
 
 // One warp, one stream.  The packed candidates and the walk-ahead results may have been produced
@@ -416,7 +468,7 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         sanitize_stream_state(sam, s, L);
         if (s != 0) r = load_rec(sam, s);
     }
-    const int nd = max(0, min(p.n_draft[b], K));
+    const int nd = (p.flags & kNoSpeculation) ? 0 : max(0, min(p.n_draft[b], K));
     RecRegs rj = root_rec();     // kTailResume: lane j fetches the record of the state reached after j + 1 drafts
     if (kMode == kTailResume && lane < nd) {
         ps = __ldcg(p.pre_state + static_cast<long long>(b) * K + lane);
@@ -434,7 +486,8 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
             const unsigned long long k = __ldcg(p.keys + row0 + j);
             p.keys[row0 + j] = 0ull;
             // no candidate at all (nothing in the row is greater than -inf): index 0, as a scan from element 0 gives
-            const int idx = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
+            int idx = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
+            if ((p.flags & kSkipUnusedRows) && j > nd) idx = -1;        // the row was not looked at
             am[h] = idx;
             p.argmax_out[row0 + j] = idx;
         }
@@ -451,7 +504,18 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         const int j = lane + 32 * h;
         if (j < K1) p.accepted[row0 + j] = (j < a) ? d : ((j == a) ? bonus : -1);
     }
-    if (lane == 0) p.n_accepted[b] = a + 1;
+    if (lane == 0) {
+        p.n_accepted[b] = a + 1;
+        if (p.counters != nullptr) {
+            // passes, committed, proposed, accepted drafts, non-empty proposals, rows looked at (Section 6.5: OTE, SHR)
+            atomicAdd(p.counters + 0, 1ull);
+            atomicAdd(p.counters + 1, static_cast<unsigned long long>(a + 1));
+            atomicAdd(p.counters + 2, static_cast<unsigned long long>(nd));
+            atomicAdd(p.counters + 3, static_cast<unsigned long long>(a));
+            atomicAdd(p.counters + 4, nd > 0 ? 1ull : 0ull);
+            atomicAdd(p.counters + 5, static_cast<unsigned long long>((p.flags & kSkipUnusedRows) ? nd + 1 : K1));
+        }
+    }
 
     if (kMode != kTailVerifyOnly) {
         if (kMode == kTailResume) {
@@ -472,7 +536,12 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
             }
         }
         walk_token(sam, bonus, s, L, r, lane);
-        const int nn = emit_draft(sam, L, r, K, p.min_match, p.next_drafts + static_cast<long long>(b) * K, lane);
+        int nn = 0;
+        if (p.flags & kNoSpeculation) {
+            if (lane < K) p.next_drafts[static_cast<long long>(b) * K + lane] = -1;
+        } else {
+            nn = emit_draft(sam, L, r, K, p.min_match, p.next_drafts + static_cast<long long>(b) * K, lane);
+        }
         if (lane == 0) {
             p.state[b] = s;
             p.matched_len[b] = L;

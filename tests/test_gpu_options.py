@@ -1,0 +1,124 @@
+"""Step options on the GPU against the oracle, tolerance 0: speculation switched off for a step
+(the adaptive switch), verification restricted to the rows a proposal uses, and the running
+OTE / SHR counters."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2512_18337_b200 as S
+import workload as W
+from tests.cuda_backend import CudaBackend, bits_to_device
+from tests.oracle_backend import OracleBackend
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KEYS = ("argmax", "accepted", "n_accepted", "state", "matched_len", "drafts", "n_draft")
+
+
+def _i32(x):
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(DEV)
+
+
+@pytest.mark.parametrize("V,pad,B,K", [(1000, 0, 5, 8), (4097, 3, 7, 4), (151936, 0, 3, 16), (151936, 8, 40, 2),
+                                       (8192 * 13 + 24, 0, 9, 5), (7, 0, 300, 1), (65536, 0, 2, 32)])
+@pytest.mark.parametrize("variant", [0, 1])
+def test_verify_skipping_unused_rows(V, pad, B, K, variant):
+    rng = np.random.default_rng(V + B + K)
+    R = B * (K + 1)
+    bits = W.f32_to_bf16_bits(rng.standard_normal((R, V + pad), dtype=np.float32))
+    if pad:
+        bits[:, V:] = 0x7F00
+    am_all = oracle.argmax_batch(bits, V=V, threads=oracle.host_threads()).reshape(B, K + 1)
+    n_draft = rng.integers(-1, K + 2, size=B).astype(np.int32)          # out-of-range counts are clamped
+    n_draft[0] = 0
+    nd = np.clip(n_draft, 0, K)
+    drafts = np.where(rng.random((B, K)) < 0.8, am_all[:, :K], rng.integers(0, V, size=(B, K))).astype(np.int32)
+    acc_o, nacc_o = oracle.accept_batch(drafts, nd, am_all)
+    lg = bits_to_device(bits)
+    outs = [torch.full(s, -9, dtype=torch.int32, device=DEV) for s in ((B, K + 1), (B, K + 1), (B,))]
+    cnt = torch.zeros(S.SAM_N_COUNTERS, dtype=torch.int64, device=DEV)
+    wsb = S.sam_workspace_bytes(B, K)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
+    S.sam_workspace_init(ws, wsb)
+    S.sam_set_argmax_variant(variant)
+    try:
+        for _ in range(2):
+            S.sam_verify_ex(lg, V + pad, B, K, V, _i32(drafts), _i32(n_draft), *outs,
+                            S.SAM_STEP_SKIP_UNUSED_ROWS, cnt, ws, wsb)
+        torch.cuda.synchronize()
+    finally:
+        S.sam_set_argmax_variant(0)
+    am, acc, nacc = (o.cpu().numpy() for o in outs)
+    used = np.arange(K + 1)[None, :] <= nd[:, None]
+    assert (am[used] == am_all[used]).all() and (am[~used] == -1).all()
+    assert (acc == acc_o).all() and (nacc == nacc_o).all()
+    a = nacc_o - 1
+    assert cnt.cpu().numpy().tolist() == [2 * B, 2 * int(nacc_o.sum()), 2 * int(nd.sum()), 2 * int(a.sum()),
+                                          2 * int((nd > 0).sum()), 2 * int((nd + 1).sum())]
+    assert S.sam_workspace_status(ws, B, K) == 0
+
+
+@pytest.mark.parametrize("variant,skip", [(0, True), (0, False), (1, True), (2, False)])
+def test_closed_loop_with_the_adaptive_switch(variant, skip):
+    """A schedule of context lengths drives the switch: steps over the threshold run without speculation.
+    Every output of every step and the final counters equal the oracle's."""
+    cfg = W.CONFIGS[1].scaled(sessions=24, B=40, steps=14, vocab=20000)
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    noise = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+    gpu = CudaBackend(cfg, corpus, bits_to_device(noise))
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    f_g, f_o = W.ClosedLoopFeeder(cfg, scripts, rowmax), W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = f_g.prime_tokens()
+    dg, ndg = gpu.prime(toks, n)
+    do, ndo = cpu.prime(toks, n)
+    cnt_g = torch.zeros(S.SAM_N_COUNTERS, dtype=torch.int64, device=DEV)
+    cnt_o = np.zeros(6, np.int64)
+    ctx_schedule = [1000, 2000, 40000, 50000, 3000, 4000, 5000, 70000, 6000, 7000, 8000, 9000, 90000, 100]
+    off_steps = 0
+    S.sam_set_argmax_variant(variant)
+    try:
+        for t in range(cfg.steps):
+            on = S.sam_adaptive_switch(ctx_schedule[t], cfg.B, 32768, 64)
+            assert on == oracle.speculation_enabled(ctx_schedule[t], cfg.B, 32768, 64)
+            flags = (0 if on else S.SAM_STEP_NO_SPECULATION) | (S.SAM_STEP_SKIP_UNUSED_ROWS if skip else 0)
+            off_steps += not on
+            zero = np.zeros(cfg.B, np.int32)
+            ow_g = f_g.overwrites(t, dg, ndg if on else zero)
+            ow_o = f_o.overwrites(t, do, ndo if on else zero)
+            keep = np.arange(ow_g["row"].shape[0])
+            sv_g = gpu.poke(ow_g["row"], ow_g["col"], ow_g["bits"], keep)
+            sv_o = cpu.poke(ow_o["row"], ow_o["col"], ow_o["bits"], keep)
+            c = cfg
+            S.sam_step_ex(gpu.index.handle, gpu.logits, gpu.stride, c.B, c.K, c.vocab, gpu.drafts, gpu.n_draft,
+                          gpu.argmax, gpu.accepted, gpu.n_accepted, gpu.state, gpu.mlen, c.min_match,
+                          gpu.drafts, gpu.n_draft, flags, cnt_g, gpu.ws, gpu.ws_bytes)
+            torch.cuda.synchronize()
+            g = dict(argmax=gpu.argmax.cpu().numpy(), accepted=gpu.accepted.cpu().numpy(),
+                     n_accepted=gpu.n_accepted.cpu().numpy(), drafts=gpu.drafts.cpu().numpy(),
+                     n_draft=gpu.n_draft.cpu().numpy(), state=gpu.state.cpu().numpy(), matched_len=gpu.mlen.cpu().numpy())
+            o = cpu.sam.step_ex(cpu.bits, c.B, c.K, c.vocab, do, ndo, cpu.state, cpu.mlen, c.min_match, flags, cnt_o)
+            o["state"], o["matched_len"] = cpu.state.copy(), cpu.mlen.copy()
+            gpu.unpoke(ow_g["row"], ow_g["col"], sv_g)
+            cpu.unpoke(ow_o["row"], ow_o["col"], sv_o)
+            for k in KEYS:
+                assert (g[k] == o[k]).all(), (t, k)
+            f_g.advance(g["n_accepted"])
+            f_o.advance(o["n_accepted"])
+            dg, ndg, do, ndo = g["drafts"], g["n_draft"], o["drafts"], o["n_draft"]
+    finally:
+        S.sam_set_argmax_variant(0)
+    assert off_steps == 4
+    assert (cnt_g.cpu().numpy() == cnt_o).all()
+    assert cnt_o[0] == cfg.B * cfg.steps and cnt_o[3] > 0
+    assert gpu.status() == 0
+
+
+def test_flags_are_checked():
+    lib = S.binding._load()
+    assert lib.sam_verify_ex(None, 8, 1, 1, 8, None, None, None, None, None, 4, None, None, 0, None) == -1
+    assert lib.sam_adaptive_switch(10, 10, 10, 10) == 1 and lib.sam_adaptive_switch(11, 10, 10, 10) == 0
