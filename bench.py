@@ -171,6 +171,9 @@ def run_ours(args):
 
     feeder = W.ClosedLoopFeeder(stream_cfg, scripts, rowmax)
     be = CudaBackend(cfg, corpus, logits, index=index, device=device)
+    be.counters = torch.zeros(S.SAM_N_COUNTERS, dtype=torch.int64, device=device)
+    if args.skip_unused_rows:
+        be.flags |= S.SAM_STEP_SKIP_UNUSED_ROWS
     toks, n = feeder.prime_tokens()
     drafts, n_draft = be.prime(toks, n)
 
@@ -211,6 +214,8 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = S.sam_launch_count()
+    be.counters.zero_()
+    torch.cuda.synchronize()
     wall0 = time.time()
     for i in range(args.steps):
         one_step(args.warmup + i, timed_slot=i)
@@ -219,6 +224,7 @@ def run_ours(args):
         dist.barrier()
     wall = time.time() - wall0
     launches = S.sam_launch_count() - launches0
+    dev_counters = [int(x) for x in be.counters.cpu().numpy()]
     clocks = sampler.stop(wall0, wall0 + wall) if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
@@ -307,7 +313,10 @@ def run_ours(args):
 
     peak, peak_kind = measured_peaks()
     R = cfg.rows
+    rows_read_per_step = dev_counters[5] / max(1, dev_counters[0]) * cfg.B     # all rows unless rows are skipped
     alg_bytes = R * (2 * cfg.vocab + 4)
+    if args.skip_unused_rows:
+        alg_bytes = rows_read_per_step * (2 * cfg.vocab + 4)
     # dominant kernel: with one launch per step the step's event bracket IS that kernel's duration (vocabulary
     # argmax with the accept / walk / draft tail inside); with two launches per step the argmax kernel's own
     # time comes from the split measurement
@@ -347,10 +356,15 @@ def run_ours(args):
         "launches_per_step": launches_per_step, "variant": args.variant,
         "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
-                     "traffic": (NCU_DRAM_BYTES_PER_ROW * R) if NCU_DRAM_BYTES_PER_ROW else None,
+                     "traffic": (NCU_DRAM_BYTES_PER_ROW * (rows_read_per_step if args.skip_unused_rows else R)) if NCU_DRAM_BYTES_PER_ROW else None,
                      "algorithmic_bytes": alg_bytes},
         "walk": walk,
         "ote": st["ote"], "shr": st["shr"], "mean_n_draft": st["mean_n_draft"],
+        "device_counters": {"passes": dev_counters[0], "committed": dev_counters[1], "proposed": dev_counters[2],
+                            "accepted_drafts": dev_counters[3], "nonempty_proposals": dev_counters[4],
+                            "rows_read": dev_counters[5], "ote": dev_counters[1] / max(1, dev_counters[0]),
+                            "shr": dev_counters[3] / max(1, dev_counters[2])},
+        "skip_unused_rows": bool(args.skip_unused_rows), "rows_read_per_step": rows_read_per_step,
         "e2e": e2e, "clocks": clocks,
         "setup_s": {"inputs": t_inputs, "sam_build": t_build, "sam_upload": t_upload,
                     "sam_build_tokens_per_s": cfg.n_corpus / t_build,
@@ -539,6 +553,9 @@ def main():
                     help="steps run after the timed region with two kernels per step, to report each kernel's time")
     ap.add_argument("--cpu-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--skip-unused-rows", action="store_true",
+                    help="verify only rows 0..n_draft[b] of every stream (SAM_STEP_SKIP_UNUSED_ROWS); a different "
+                         "workload from the default one, which reads all B*(K+1) rows")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()

@@ -30,6 +30,8 @@ class CudaBackend:
         self.argmax = torch.full((B, K + 1), -7, **i32)
         self.accepted = torch.full((B, K + 1), -7, **i32)
         self.n_accepted = torch.zeros(B, **i32)
+        self.flags = 0              # SAM_STEP_* options used by launch_step
+        self.counters = None        # optional int64[SAM_N_COUNTERS] device tensor
         self.ws_bytes = S.sam_workspace_bytes(B, K)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         S.sam_workspace_init(self.ws, self.ws_bytes)
@@ -60,9 +62,9 @@ class CudaBackend:
     def launch_step(self):
         """Enqueue one fused step on the current stream (drafts/n_draft are updated in place)."""
         c = self.cfg
-        S.sam_step(self.index.handle, self.logits, self.stride, c.B, c.K, c.vocab, self.drafts, self.n_draft,
-                   self.argmax, self.accepted, self.n_accepted, self.state, self.mlen, c.min_match,
-                   self.drafts, self.n_draft, self.ws, self.ws_bytes)
+        S.sam_step_ex(self.index.handle, self.logits, self.stride, c.B, c.K, c.vocab, self.drafts, self.n_draft,
+                      self.argmax, self.accepted, self.n_accepted, self.state, self.mlen, c.min_match,
+                      self.drafts, self.n_draft, self.flags, self.counters, self.ws, self.ws_bytes)
 
     def status(self) -> int:
         return S.sam_workspace_status(self.ws, self.cfg.B, self.cfg.K)
