@@ -536,6 +536,88 @@ def run_growing(args):
     }))
 
 
+# ----------------------------------------------------------------------------- vocabulary-parallel verification
+def run_vocab_parallel(args):
+    """The closed loop with the vocabulary split into column shards (tensor-parallel output layer).
+    Under torchrun every rank owns one shard of the same logits and the per-row words are combined by one
+    NCCL MAX all-reduce; on a single process all shards are reduced one after the other on the one GPU and
+    merged there.  Prints its own JSON line."""
+    import torch
+    import torch.distributed as dist
+    import paper_2512_18337_b200 as S
+    from paper_2512_18337_b200.build import build
+    from paper_2512_18337_b200.parallel import reduce_argmax_keys, shard_bounds
+    from tests.cuda_backend import CudaBackend
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    device = f"cuda:{local_rank}"
+    torch.cuda.set_device(device)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    shards = world if world > 1 else args.vocab_shards
+    mine = [rank] if world > 1 else list(range(shards))
+    cfg = W.CONFIGS[args.config].scaled(steps=args.warmup + args.steps + 1)
+    corpus, logits, rowmax = make_inputs_gpu(cfg, device)       # same seed on every rank: same logits
+    scripts = W.make_scripts(cfg, corpus)
+    feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    be = CudaBackend(cfg, corpus, logits, device=device)
+    toks, n = feeder.prime_tokens()
+    drafts, n_draft = be.prime(toks, n)
+    R, c = cfg.rows, cfg
+    keys = [torch.zeros(R + 1, dtype=torch.int64, device=device) for _ in mine]
+    merged = torch.zeros(R, dtype=torch.int64, device=device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    tokens = 0
+    for t in range(args.warmup + args.steps):
+        ow = feeder.overwrites(t, drafts, n_draft)
+        saved = be.poke(ow["row"], ow["col"], ow["bits"], np.arange(ow["row"].shape[0]))
+        i = t - args.warmup
+        if i >= 0:
+            torch.cuda._sleep(args.presleep_cycles)
+            ev[i][0].record()
+        for k, r in zip(keys, mine):
+            lo, hi = shard_bounds(c.vocab, r, shards)
+            S.sam_argmax_partial(be.logits.data_ptr() + 2 * lo, be.stride, R, hi - lo, lo, k)
+        if world > 1:
+            reduce_argmax_keys(keys[0], R)
+            words = keys[0]
+        else:
+            merged.copy_(keys[0][:R])
+            for k in keys[1:]:
+                torch.maximum(merged, k[:R], out=merged)
+            words = merged
+        S.sam_step_from_keys(be.index.handle, words, c.B, c.K, be.drafts, be.n_draft, be.argmax, be.accepted,
+                             be.n_accepted, be.state, be.mlen, c.min_match, be.drafts, be.n_draft)
+        if i >= 0:
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        n_acc = be.n_accepted.cpu().numpy()
+        drafts, n_draft = be.drafts.cpu().numpy(), be.n_draft.cpu().numpy()
+        be.unpoke(ow["row"], ow["col"], saved)
+        feeder.advance(n_acc)
+        if i >= 0:
+            tokens += int(n_acc.sum())
+    ms = float(sum(a.elapsed_time(b) for a, b in ev))
+    _, ms = reduce_over_ranks(0, ms, world, device)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC + "_vocab_parallel", "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "dtype": "bf16 compare / int32", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": c.B, "K": c.K, "V": c.vocab, "vocab_shards": shards,
+                       "shards_reduced_per_gpu": len(mine),
+                       "timing": "CUDA events around sam_argmax_partial (per shard) + merge + sam_step_from_keys"},
+            "bytes_reduced_per_gpu_per_step": sum(R * 2 * (shard_bounds(c.vocab, r, shards)[1] - shard_bounds(c.vocab, r, shards)[0]) for r in mine),
+            "allreduce_bytes_per_step": R * 8 if world > 1 else 0,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -556,6 +638,9 @@ def main():
     ap.add_argument("--skip-unused-rows", action="store_true",
                     help="verify only rows 0..n_draft[b] of every stream (SAM_STEP_SKIP_UNUSED_ROWS); a different "
                          "workload from the default one, which reads all B*(K+1) rows")
+    ap.add_argument("--vocab-shards", type=int, default=0,
+                    help="> 0: time verification over a column-sharded vocabulary (one shard per rank under torchrun; "
+                         "all shards one after the other on a single GPU); prints a separate JSON line")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()
@@ -564,6 +649,8 @@ def main():
         run_reference(args)
     elif args.growing:
         run_growing(args)
+    elif args.vocab_shards > 0:
+        run_vocab_parallel(args)
     else:
         run_ours(args)
 

@@ -191,6 +191,30 @@ int sam_step_ex(const sam_index* idx,
                 uint32_t flags, int64_t* counters,
                 void* workspace, int64_t workspace_bytes, void* cuda_stream);
 
+/* Verification in two halves, for a vocabulary that is split over several GPUs (the target model's
+ * output layer under tensor parallelism; the paper runs its models with TP 2-8 but does not discuss
+ * verification there - this is the natural composition).
+ *
+ * sam_argmax_partial reduces rows x V logits that are columns v_offset .. v_offset+V-1 of the full
+ * vocabulary and leaves one 64-bit word per row in keys: 0 when the shard holds nothing greater than
+ * -inf, otherwise a packed (value, index) whose signed 64-bit order is "greater value first, then
+ * smaller GLOBAL index".  The elementwise maximum of the shards' words - one MAX all-reduce of
+ * rows x 8 bytes over NCCL, or any other route - is therefore the word of the full row, ties and all.
+ *   keys   device, int64[rows + 1], 8-byte aligned; zeroed by this call; keys[rows] is a status word
+ *          (0 = fine, see sam_workspace_status) and should be left out of the reduction
+ *   A row whose GLOBAL element 0 is NaN yields index 0 (only the shard with v_offset = 0 can tell).
+ * sam_step_from_keys takes the reduced words (device, int64[B*(K+1)]; they are re-zeroed), decodes them
+ * into argmax_out and then does what sam_step does after its argmax: accept, follow the committed
+ * tokens from (state, matched_len), emit the next draft.
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_CUDA. */
+int sam_argmax_partial(const void* logits_bf16, int64_t row_stride_elems, int64_t rows, int32_t V, int32_t v_offset,
+                       int64_t* keys, void* cuda_stream);
+int sam_step_from_keys(const sam_index* idx, int64_t* keys, int32_t B, int32_t K,
+                       const int32_t* drafts, const int32_t* n_draft,
+                       int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                       int32_t* state, int32_t* matched_len, int32_t min_match,
+                       int32_t* next_drafts, int32_t* next_n_draft, void* cuda_stream);
+
 /* The adaptive switch itself (Section 5.4.3; Algorithm 3 step 4): 1 = keep speculating, 0 = fall back
  * to plain decoding because the context length or the batch size exceeds its threshold.  The
  * thresholds are deployment-specific ("empirically determined" in the paper); a host-side helper,

@@ -41,6 +41,8 @@ _SIGNATURES = {
     "sam_step_ex": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                               _vp, _vp, _i32, _vp, _vp, C.c_uint32, _vp, _vp, _i64, _vp]),
     "sam_adaptive_switch": (C.c_int, [_i64, _i64, _i64, _i64]),
+    "sam_argmax_partial": (C.c_int, [_vp, _i64, _i64, _i32, _i32, _vp, _vp]),
+    "sam_step_from_keys": (C.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "sam_verify_static": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
@@ -277,6 +279,20 @@ def sam_step_ex(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out
                                _dev(argmax_out), _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len),
                                min_match, _dev(next_drafts), _dev(next_n_draft), flags, _dev(counters),
                                _dev(workspace), workspace_bytes, _stream(stream)), "sam_step_ex")
+
+
+def sam_argmax_partial(logits, row_stride, rows, V, v_offset, keys, stream=None):
+    """Packed per-row argmax words of a vocabulary shard (columns v_offset.. of the full vocabulary);
+    keys: int64[rows + 1] device tensor (last word = status)."""
+    _check(_load().sam_argmax_partial(_dev(logits), row_stride, rows, V, v_offset, _dev(keys), _stream(stream)),
+           "sam_argmax_partial")
+
+
+def sam_step_from_keys(handle, keys, B, K, drafts, n_draft, argmax_out, accepted, n_accepted,
+                       state, matched_len, min_match, next_drafts, next_n_draft, stream=None):
+    _check(_load().sam_step_from_keys(handle, _dev(keys), B, K, _dev(drafts), _dev(n_draft), _dev(argmax_out),
+                                      _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len), min_match,
+                                      _dev(next_drafts), _dev(next_n_draft), _stream(stream)), "sam_step_from_keys")
 
 
 def sam_adaptive_switch(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:

@@ -561,6 +561,36 @@ int sam_step(const sam_index* idx,
                        workspace, workspace_bytes, cuda_stream);
 }
 
+int sam_argmax_partial(const void* logits_bf16, int64_t row_stride_elems, int64_t rows, int32_t V, int32_t v_offset,
+                       int64_t* keys, void* cuda_stream) {
+    if (rows < 0 || V < 1 || row_stride_elems < V || v_offset < 0 || static_cast<int64_t>(v_offset) + V > (int64_t(1) << 31) - 1)
+        return SAM_ERR_INVALID_ARG;
+    if (rows == 0) return SAM_OK;
+    if (!logits_bf16 || !keys || !aligned(logits_bf16, 2) || !aligned(keys, 8)) return SAM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SAM_CUDA(cudaMemsetAsync(keys, 0, static_cast<size_t>(rows + 1) * 8, st));     // the last word is the status word
+    const RowMap rm{nullptr, nullptr, v_offset};
+    return launch_argmax(logits_bf16, row_stride_elems, rows, V, reinterpret_cast<unsigned long long*>(keys),
+                         reinterpret_cast<int*>(keys + rows), st, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, &rm);
+}
+
+int sam_step_from_keys(const sam_index* idx, int64_t* keys, int32_t B, int32_t K,
+                       const int32_t* drafts, const int32_t* n_draft,
+                       int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                       int32_t* state, int32_t* matched_len, int32_t min_match,
+                       int32_t* next_drafts, int32_t* next_n_draft, void* cuda_stream) {
+    if (!idx || B < 0 || K < 1 || K > SAM_K_MAX || min_match < 1) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!keys || !aligned(keys, 8) || !drafts || !n_draft || !argmax_out || !accepted || !n_accepted || !state ||
+        !matched_len || !next_drafts || !next_n_draft)
+        return SAM_ERR_INVALID_ARG;
+    const AcceptArgs aa{nullptr, 0, B, K, drafts, n_draft, argmax_out, accepted, n_accepted,
+                        reinterpret_cast<unsigned long long*>(keys), state, matched_len, min_match, next_drafts,
+                        next_n_draft, nullptr, nullptr, 0u, nullptr};
+    return launch_accept<kTailFullWalk>(idx->dev, aa, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_context_len, int64_t max_batch_size) {
     return (context_len > max_context_len || batch_size > max_batch_size) ? 0 : 1;
 }

@@ -122,3 +122,58 @@ def test_flags_are_checked():
     lib = S.binding._load()
     assert lib.sam_verify_ex(None, 8, 1, 1, 8, None, None, None, None, None, 4, None, None, 0, None) == -1
     assert lib.sam_adaptive_switch(10, 10, 10, 10) == 1 and lib.sam_adaptive_switch(11, 10, 10, 10) == 0
+
+
+@pytest.mark.parametrize("shards,multiple", [(4, 8), (3, 1), (8, 8)])
+def test_vocabulary_shards_merge_to_the_full_row(shards, multiple):
+    """The vocabulary split into column shards (aligned ones take the bulk-copy kernel, odd ones the
+    direct-load kernel): per-shard words, elementwise maximum, then accept + walk + draft from the
+    merged words equal the oracle's step on the whole rows - ties across shards and NaN rows included."""
+    from paper_2512_18337_b200.parallel import shard_bounds
+    cfg = W.CONFIGS[1].scaled(sessions=16, B=12, steps=4, vocab=50257)
+    c = cfg
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    noise = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+    # exact ties that straddle shards, and NaNs at the start of the row and of a later shard
+    noise[1, [100, 40000]] = 0x4140
+    noise[2, [49000, 7]] = 0x4140
+    noise[3, 0] = 0x7FC0
+    noise[4, shard_bounds(c.vocab, 1, shards, multiple)[0]] = 0x7FC0
+    gpu = CudaBackend(cfg, corpus, bits_to_device(noise))
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    f_g, f_o = W.ClosedLoopFeeder(cfg, scripts, rowmax), W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = f_g.prime_tokens()
+    dg, ndg = gpu.prime(toks, n)
+    do, ndo = cpu.prime(toks, n)
+    R = c.B * (c.K + 1)
+    for t in range(c.steps):
+        ow = f_g.overwrites(t, dg, ndg)
+        f_o.overwrites(t, do, ndo)
+        keep = np.arange(ow["row"].shape[0])
+        sv_g = gpu.poke(ow["row"], ow["col"], ow["bits"], keep)
+        sv_o = cpu.poke(ow["row"], ow["col"], ow["bits"], keep)
+        merged = torch.zeros(R, dtype=torch.int64, device=DEV)
+        for r in range(shards):
+            lo, hi = shard_bounds(c.vocab, r, shards, multiple)
+            keys = torch.full((R + 1,), -1, dtype=torch.int64, device=DEV)
+            S.sam_argmax_partial(gpu.logits.data_ptr() + 2 * lo, gpu.stride, R, hi - lo, lo, keys)
+            torch.cuda.synchronize()
+            assert int(keys[R]) == 0
+            merged = torch.maximum(merged, keys[:R])
+        S.sam_step_from_keys(gpu.index.handle, merged, c.B, c.K, gpu.drafts, gpu.n_draft, gpu.argmax, gpu.accepted,
+                             gpu.n_accepted, gpu.state, gpu.mlen, c.min_match, gpu.drafts, gpu.n_draft)
+        torch.cuda.synchronize()
+        assert int(merged.abs().sum()) == 0                      # the words are handed back zeroed
+        g = dict(argmax=gpu.argmax.cpu().numpy(), accepted=gpu.accepted.cpu().numpy(),
+                 n_accepted=gpu.n_accepted.cpu().numpy(), drafts=gpu.drafts.cpu().numpy(),
+                 n_draft=gpu.n_draft.cpu().numpy(), state=gpu.state.cpu().numpy(), matched_len=gpu.mlen.cpu().numpy())
+        o = cpu.step(do, ndo)
+        gpu.unpoke(ow["row"], ow["col"], sv_g)
+        cpu.unpoke(ow["row"], ow["col"], sv_o)
+        for k in KEYS:
+            assert (g[k] == o[k]).all(), (t, k)
+        f_g.advance(g["n_accepted"])
+        f_o.advance(o["n_accepted"])
+        dg, ndg, do, ndo = g["drafts"], g["n_draft"], o["drafts"], o["n_draft"]
