@@ -246,3 +246,40 @@ def accept_batch(drafts: np.ndarray, n_draft: np.ndarray, argmax: np.ndarray):
     n_acc = np.empty(B, np.int32)
     _load().oracle_accept_batch(B, K, _i32(drafts), _i32(n_draft), _i32(argmax), _i32(acc), _i32(n_acc))
     return acc, n_acc
+
+
+def multi_draft(members, slots, weights, state, matched_len, new_tokens, n_new, K, min_match):
+    """Composite drafting over several automata (Section 5.4.2: the session's own context plus the
+    top-K retrieved contexts, "the similarity scores determine the weights of each SAM").
+
+    The paper names the ingredients but not the rule; the reading taken here: every stream b has M
+    slots, slot m naming one member automaton (slots[b, m], -1 = empty) with a weight; each slot
+    keeps its own (state, matched_len) and follows the new tokens in its own automaton; the draft
+    comes from the slot with the largest weight * matched_len (float32 product) among the slots
+    whose match reaches min_match, the lowest slot winning ties; no such slot, no draft.
+
+    members: list of OracleSAM; slots [B, M] int32; weights [B, M] float32; state, matched_len
+    [B, M] int32 (updated in place); new_tokens [B, ld], n_new [B].
+    Returns (drafts [B, K], n_draft [B], chosen [B] slot or -1)."""
+    B, M = slots.shape
+    drafts = np.full((B, K), -1, np.int32)
+    n_draft = np.zeros(B, np.int32)
+    chosen = np.full(B, -1, np.int32)
+    for b in range(B):
+        best_score, best_m = None, -1
+        for m in range(M):
+            if slots[b, m] < 0:
+                continue
+            sam = members[int(slots[b, m])]
+            s, L = sam.walk(int(state[b, m]), int(matched_len[b, m]), new_tokens[b, :max(0, int(n_new[b]))])
+            state[b, m], matched_len[b, m] = s, L
+            if L < min_match:
+                continue
+            score = np.float32(weights[b, m]) * np.float32(L)
+            if best_score is None or score > best_score:
+                best_score, best_m = score, m
+        if best_m >= 0:
+            sam = members[int(slots[b, best_m])]
+            d, nd = sam.draft(int(state[b, best_m]), int(matched_len[b, best_m]), K, min_match)
+            drafts[b], n_draft[b], chosen[b] = d, nd, best_m
+    return drafts, n_draft, chosen
