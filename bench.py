@@ -618,6 +618,82 @@ def run_vocab_parallel(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- composite drafting
+def run_multi(args):
+    """Closed loop with composite drafting: the corpus of the chosen workload is split into M member
+    automata (sessions dealt round-robin), every stream holds all M with weights from {0.5, 1, 1.5}; a step is
+    sam_verify followed by sam_multi_draft on the accepted tokens.  Prints its own JSON line."""
+    import torch
+    import paper_2512_18337_b200 as S
+    from paper_2512_18337_b200.build import build
+
+    device = "cuda:0"
+    torch.cuda.set_device(device)
+    build()
+    M = args.multi
+    cfg = W.CONFIGS[args.config].scaled(steps=args.warmup + args.steps + 1)
+    corpus, logits, rowmax = make_inputs_gpu(cfg, device)
+    scripts = W.make_scripts(cfg, corpus)
+    ln = cfg.session_len + 1
+    padded = np.concatenate([corpus, [cfg.separator]]).reshape(cfg.sessions, ln)
+    t0 = time.time()
+    members = [S.SamIndex(np.ascontiguousarray(padded[m::M]).reshape(-1)[:-1], [cfg.separator], device=device) for m in range(M)]
+    t_build = time.time() - t0
+    sset = S.SamSet(members, device=device)
+    B, K, V = cfg.B, cfg.K, cfg.vocab
+    rng = np.random.default_rng(cfg.seed)
+    i32 = dict(dtype=torch.int32, device=device)
+    slots = torch.arange(M, **i32).repeat(B, 1).contiguous()
+    weights = torch.from_numpy(rng.choice(np.array([0.5, 1.0, 1.5], np.float32), size=(B, M))).to(device)
+    st, ml = torch.zeros((B, M), **i32), torch.zeros((B, M), **i32)
+    drafts, n_draft, chosen = torch.full((B, K), -1, **i32), torch.zeros(B, **i32), torch.zeros(B, **i32)
+    am, acc, nacc = torch.zeros((B, K + 1), **i32), torch.zeros((B, K + 1), **i32), torch.zeros(B, **i32)
+    wsb = S.sam_workspace_bytes(B, K)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=device)
+    S.sam_workspace_init(ws, wsb)
+    raw = logits.view(torch.int16)
+    feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = feeder.prime_tokens()
+    S.sam_multi_draft(sset.handle, B, M, slots, weights, st, ml, torch.from_numpy(toks).to(device), toks.shape[1],
+                      torch.from_numpy(n).to(device), K, cfg.min_match, drafts, n_draft, chosen)
+    torch.cuda.synchronize()
+    ev = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(args.steps)]
+    tokens = drafted = 0
+    for t in range(args.warmup + args.steps):
+        ow = feeder.overwrites(t, drafts.cpu().numpy(), n_draft.cpu().numpy())
+        r, c = torch.from_numpy(ow["row"]).to(device), torch.from_numpy(ow["col"]).to(device)
+        saved = raw[r, c].clone()
+        raw[r, c] = torch.from_numpy(ow["bits"].view(np.int16)).to(device)
+        i = t - args.warmup
+        if i >= 0:
+            drafted += int(n_draft.sum())
+            torch.cuda._sleep(args.presleep_cycles)
+            ev[i][0].record()
+        S.sam_verify(logits, V, B, K, V, drafts, n_draft, am, acc, nacc, ws, wsb)
+        if i >= 0:
+            ev[i][1].record()
+        S.sam_multi_draft(sset.handle, B, M, slots, weights, st, ml, acc, K + 1, nacc, K, cfg.min_match, drafts, n_draft, chosen)
+        if i >= 0:
+            ev[i][2].record()
+        torch.cuda.synchronize()
+        raw[r, c] = saved
+        n_acc = nacc.cpu().numpy()
+        feeder.advance(n_acc)
+        if i >= 0:
+            tokens += int(n_acc.sum())
+    ms = float(sum(e[0].elapsed_time(e[2]) for e in ev))
+    ms_multi = float(sum(e[1].elapsed_time(e[2]) for e in ev))
+    print(json.dumps({
+        "metric": METRIC + "_composite", "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "dtype": "bf16 compare / int32",
+        "data": "synthetic",
+        "config": {"workload": cfg.name + f" split into {M} member automata, every stream holds all {M}", "B": B, "K": K,
+                   "V": V, "timing": "CUDA events around sam_verify + sam_multi_draft"},
+        "multi_draft_kernel_ms": ms_multi / args.steps, "slot_walks_per_s": B * M * args.steps / (ms_multi / 1e3),
+        "mean_n_draft": drafted / (B * args.steps), "ote": tokens / (B * args.steps), "members_build_s": t_build,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -641,6 +717,8 @@ def main():
     ap.add_argument("--vocab-shards", type=int, default=0,
                     help="> 0: time verification over a column-sharded vocabulary (one shard per rank under torchrun; "
                          "all shards one after the other on a single GPU); prints a separate JSON line")
+    ap.add_argument("--multi", type=int, default=0,
+                    help="> 0: closed loop with composite drafting over that many member automata (1..8); separate JSON line")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()
@@ -649,6 +727,8 @@ def main():
         run_reference(args)
     elif args.growing:
         run_growing(args)
+    elif args.multi > 0:
+        run_multi(args)
     elif args.vocab_shards > 0:
         run_vocab_parallel(args)
     else:

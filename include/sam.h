@@ -318,6 +318,41 @@ int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_i
  * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_CUDA. */
 int sam_renormalize(const sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream);
 
+/* ---------------------------------------------------------------- composite drafting */
+
+/* Drafting from several automata at once (Section 5.4.2; Algorithm 3 step 1: the automaton of the
+ * current session is combined with those of the top-K retrieved contexts, "the similarity scores
+ * determine the weights of each SAM").  The paper does not define the combination; the rule here:
+ * every stream has M slots, each naming one member index and carrying a weight; each slot keeps its
+ * own (state, matched_len) and follows the new tokens in its own automaton; the draft is emitted by
+ * the slot with the largest weight * matched_len (float32 product) among the slots whose match
+ * reaches min_match, the lowest slot winning ties; if no slot qualifies there is no draft.
+ * Retrieval and similarity scoring are the caller's business: slots and weights are inputs.
+ *
+ * sam_set_create copies the device views of n_members uploaded indexes into a caller-owned device
+ * table (device_buf, at least sam_set_bytes(n_members), 16-byte aligned); the member handles must
+ * outlive the set.  After a member has grown (sam_sync), sam_set_refresh copies the views again.
+ *
+ * sam_multi_draft: as sam_draft, with per-slot state:
+ *   slots        device [B, M] int32, member number or -1 for an empty slot;  1 <= M <= 8
+ *   weights      device [B, M] float32
+ *   state, matched_len   device [B, M] int32, in/out (a new slot starts at (0, 0))
+ *   new_tokens, ld, n_new, K, min_match, drafts, n_draft   as in sam_draft (shared by all slots)
+ *   chosen       device [B] int32: the slot that drafted, or -1
+ * Verification needs nothing new: sam_verify on the emitted drafts, then sam_multi_draft with
+ * new_tokens = accepted, n_new = n_accepted.
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_SMALL, SAM_ERR_NOT_UPLOADED, SAM_ERR_NOMEM, SAM_ERR_CUDA. */
+typedef struct sam_set sam_set;
+int64_t sam_set_bytes(int32_t n_members);
+int sam_set_create(const sam_index* const* members, int32_t n_members, void* device_buf, int64_t bytes,
+                   void* cuda_stream, sam_set** out);
+int sam_set_refresh(sam_set* set, void* cuda_stream);
+void sam_set_free(sam_set* set);
+int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slots, const float* weights,
+                    int32_t* state, int32_t* matched_len, const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
+                    int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, int32_t* chosen,
+                    void* cuda_stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 
 /* Per-kernel device timing of sam_verify / sam_step (measurement aid; the paper has no

@@ -198,6 +198,7 @@ osam *oracle_sam_build(const int32_t *corpus, int64_t n)
 int32_t oracle_renormalize(const osam *a, int32_t state, int32_t matched_len)
 {
     int32_t s = state;
+    if (s < 0 || s >= a->n_states) return state;   /* not a state of this automaton: left alone */
     while (s != 0 && matched_len <= a->st[a->st[s].link].len) s = a->st[s].link;
     return s;
 }

@@ -41,6 +41,11 @@ _SIGNATURES = {
     "sam_step_ex": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                               _vp, _vp, _i32, _vp, _vp, C.c_uint32, _vp, _vp, _i64, _vp]),
     "sam_adaptive_switch": (C.c_int, [_i64, _i64, _i64, _i64]),
+    "sam_set_bytes": (_i64, [_i32]),
+    "sam_set_create": (C.c_int, [_vp, _i32, _vp, _i64, _vp, C.POINTER(_vp)]),
+    "sam_set_refresh": (C.c_int, [_vp, _vp]),
+    "sam_set_free": (None, [_vp]),
+    "sam_multi_draft": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp]),
     "sam_argmax_partial": (C.c_int, [_vp, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sam_step_from_keys": (C.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "sam_verify_static": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -293,6 +298,42 @@ def sam_step_from_keys(handle, keys, B, K, drafts, n_draft, argmax_out, accepted
     _check(_load().sam_step_from_keys(handle, _dev(keys), B, K, _dev(drafts), _dev(n_draft), _dev(argmax_out),
                                       _dev(accepted), _dev(n_accepted), _dev(state), _dev(matched_len), min_match,
                                       _dev(next_drafts), _dev(next_n_draft), _stream(stream)), "sam_step_from_keys")
+
+
+class SamSet:
+    """A table of uploaded indexes for composite drafting (owns the small device table)."""
+
+    def __init__(self, indexes, device="cuda:0", stream=None):
+        import torch
+        self.indexes = list(indexes)                      # keeps the members alive
+        n = len(self.indexes)
+        nbytes = _load().sam_set_bytes(n)
+        self.table = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        arr = (_vp * n)(*[ix.handle for ix in self.indexes])
+        h = _vp()
+        _check(_load().sam_set_create(arr, n, _dev(self.table), nbytes, _stream(stream), C.byref(h)), "sam_set_create")
+        self.handle = h.value
+
+    def refresh(self, stream=None):
+        _check(_load().sam_set_refresh(self.handle, _stream(stream)), "sam_set_refresh")
+
+    def close(self):
+        h, self.handle = self.handle, None
+        if h:
+            _load().sam_set_free(h)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def sam_multi_draft(set_handle, B, M, slots, weights, state, matched_len, new_tokens, ld, n_new, K, min_match,
+                    drafts, n_draft, chosen, stream=None):
+    _check(_load().sam_multi_draft(set_handle, B, M, _dev(slots), _dev(weights), _dev(state), _dev(matched_len),
+                                   _dev(new_tokens), ld, _dev(n_new), K, min_match, _dev(drafts), _dev(n_draft),
+                                   _dev(chosen), _stream(stream)), "sam_multi_draft")
 
 
 def sam_adaptive_switch(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:

@@ -338,6 +338,11 @@ int upload_growing(sam_index* idx, void* device_buf, cudaStream_t st) {
 
 }  // namespace
 
+struct sam_set {
+    std::vector<const sam_index*> members;
+    void* device_buf = nullptr;      // caller-owned table of DeviceSam
+};
+
 extern "C" {
 
 int sam_build(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep, sam_index** out) {
@@ -589,6 +594,61 @@ int sam_step_from_keys(const sam_index* idx, int64_t* keys, int32_t B, int32_t K
                         reinterpret_cast<unsigned long long*>(keys), state, matched_len, min_match, next_drafts,
                         next_n_draft, nullptr, nullptr, 0u, nullptr};
     return launch_accept<kTailFullWalk>(idx->dev, aa, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int64_t sam_set_bytes(int32_t n_members) {
+    if (n_members < 1) return SAM_ERR_INVALID_ARG;
+    return (static_cast<int64_t>(n_members) * static_cast<int64_t>(sizeof(DeviceSam)) + 255) & ~int64_t(255);
+}
+
+int sam_set_refresh(sam_set* set, void* cuda_stream) {
+    if (!set || !set->device_buf) return SAM_ERR_INVALID_ARG;
+    std::vector<DeviceSam> table(set->members.size());
+    for (size_t i = 0; i < set->members.size(); ++i) {
+        if (!set->members[i]->device_buf) return SAM_ERR_NOT_UPLOADED;
+        table[i] = set->members[i]->dev;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SAM_CUDA(cudaMemcpyAsync(set->device_buf, table.data(), table.size() * sizeof(DeviceSam), cudaMemcpyHostToDevice, st));
+    return SAM_OK;
+}
+
+int sam_set_create(const sam_index* const* members, int32_t n_members, void* device_buf, int64_t bytes,
+                   void* cuda_stream, sam_set** out) {
+    if (!members || n_members < 1 || !device_buf || !out || !aligned(device_buf, 16)) return SAM_ERR_INVALID_ARG;
+    if (bytes < sam_set_bytes(n_members)) return SAM_ERR_TOO_SMALL;
+    for (int32_t i = 0; i < n_members; ++i)
+        if (!members[i]) return SAM_ERR_INVALID_ARG;
+    sam_set* set = new (std::nothrow) sam_set();
+    if (!set) return SAM_ERR_NOMEM;
+    set->members.assign(members, members + n_members);
+    set->device_buf = device_buf;
+    const int rc = sam_set_refresh(set, cuda_stream);
+    if (rc != SAM_OK) {
+        delete set;
+        return rc;
+    }
+    *out = set;
+    return SAM_OK;
+}
+
+void sam_set_free(sam_set* set) { delete set; }
+
+int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slots, const float* weights,
+                    int32_t* state, int32_t* matched_len, const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
+                    int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, int32_t* chosen,
+                    void* cuda_stream) {
+    if (!set || B < 0 || M < 1 || M > kMaxSlots || K < 1 || K > SAM_K_MAX || min_match < 1 || ld < 0)
+        return SAM_ERR_INVALID_ARG;
+    if (B == 0) return SAM_OK;
+    if (!slots || !weights || !state || !matched_len || !n_new || !drafts || !n_draft || !chosen || (ld > 0 && !new_tokens))
+        return SAM_ERR_INVALID_ARG;
+    multi_draft_kernel<<<static_cast<unsigned>(B), 32 * M, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<const DeviceSam*>(set->device_buf), static_cast<int>(set->members.size()), B, M, slots, weights,
+        state, matched_len, new_tokens, ld, n_new, K, min_match, drafts, n_draft, chosen);
+    SAM_CUDA(cudaGetLastError());
+    ++g_launches;
+    return SAM_OK;
 }
 
 int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_context_len, int64_t max_batch_size) {

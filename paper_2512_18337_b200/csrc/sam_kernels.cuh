@@ -164,6 +164,72 @@ draft_kernel(DeviceSam sam, int B, int* __restrict__ state, int* __restrict__ ma
     }
 }
 
+// Composite drafting over several automata (Section 5.4.2: the session's context plus the retrieved
+// contexts, weighted by similarity).  One CTA per stream, one warp per slot: every slot follows the
+// new tokens in its own automaton from its own (state, matched_len); the draft comes from the slot
+// with the largest weight * matched_len (float32) among those that reach min_match, the lowest slot
+// winning ties.
+constexpr int kMaxSlots = 8;
+
+__global__ void __launch_bounds__(32 * kMaxSlots)
+multi_draft_kernel(const DeviceSam* __restrict__ table, int n_members, int B, int M,
+                   const int* __restrict__ slots, const float* __restrict__ weights,
+                   int* __restrict__ state, int* __restrict__ matched_len,
+                   const int* __restrict__ new_tokens, int ld, const int* __restrict__ n_new,
+                   int K, int min_match, int* __restrict__ drafts, int* __restrict__ n_draft,
+                   int* __restrict__ chosen) {
+    __shared__ float score[kMaxSlots];
+    __shared__ int ok[kMaxSlots];
+    __shared__ int winner;
+    const int b = blockIdx.x;
+    const int m = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long at = static_cast<long long>(b) * M + m;
+    const int member = slots[at];
+    const bool live = member >= 0 && member < n_members;
+    int s = 0, L = 0;
+    RecRegs r = root_rec();
+    DeviceSam sam;
+    if (live) {
+        sam = table[member];
+        s = state[at];
+        L = matched_len[at];
+        sanitize_stream_state(sam, s, L);
+        if (s != 0) r = load_rec(sam, s);
+        const int n = max(0, min(n_new[b], ld));
+        const int* row = new_tokens + static_cast<long long>(b) * ld;
+        for (int base = 0; base < n; base += 32) {
+            const int mine = (base + lane < n) ? __ldg(row + base + lane) : -1;
+            const int cnt = min(32, n - base);
+            for (int t = 0; t < cnt; ++t) walk_token(sam, __shfl_sync(kFull, mine, t), s, L, r, lane);
+        }
+        if (lane == 0) {
+            state[at] = s;
+            matched_len[at] = L;
+        }
+    }
+    if (lane == 0) {
+        ok[m] = live && L >= min_match;
+        score[m] = live ? weights[at] * static_cast<float>(L) : 0.0f;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int w = -1;
+        float best = 0.0f;
+        for (int q = 0; q < M; ++q)
+            if (ok[q] && (w < 0 || score[q] > best)) { w = q; best = score[q]; }
+        winner = w;
+        chosen[b] = w;
+        if (w < 0) n_draft[b] = 0;
+    }
+    __syncthreads();
+    if (winner == m) {
+        const int nd = emit_draft(sam, L, r, K, min_match, drafts + static_cast<long long>(b) * K, lane);
+        if (lane == 0) n_draft[b] = nd;
+    } else if (winner < 0 && m == 0 && lane < K) {
+        drafts[static_cast<long long>(b) * K + lane] = -1;
+    }
+}
+
 // Walk-ahead along the draft.  While the logits of a step are still being reduced, spare warps
 // follow the automaton over each stream's DRAFT tokens and record the (state, matched_len)
 // reached after every prefix.  Whatever prefix the verification later accepts, the walk over it
