@@ -189,6 +189,8 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
     int* queue = reinterpret_cast<int*>(smem_raw + kBulkQueueOff);
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem_raw + kBulkCandOff);   // [kRowSlots][warps]
 
+    // the accept kernel may be scheduled now; it waits for this grid before it reads any result
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     // with a row list the number of rows is only known on the device, and a CTA's share may be empty

@@ -189,9 +189,20 @@ template <int kMode>
 int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st) {
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((a.B + warps - 1) / warps);
-    accept_kernel<kMode><<<grid, warps * 32, 0, st>>>(sam, a);
+    // launched as a programmatic dependent of the kernel before it in the stream (the argmax kernel): its
+    // blocks are placed, and load what does not depend on that kernel, while that kernel is still running
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    SAM_CUDA(cudaLaunchKernelEx(&cfg, accept_kernel<kMode>, sam, a));
     ++g_launches;
-    SAM_CUDA(cudaGetLastError());
     return SAM_OK;
 }
 

@@ -433,6 +433,8 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
 __global__ void __launch_bounds__(kArgmaxThreads)
 argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
                      int tiles_per_row, unsigned long long* __restrict__ keys, RowMap rm) {
+    // the accept kernel may be scheduled now; it waits for this grid before it reads any result
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (rm.list != nullptr) R = __ldg(rm.n_rows);
     const long long total = R * tiles_per_row;
     const long long t0 = total * blockIdx.x / gridDim.x;
@@ -520,7 +522,9 @@ struct AcceptArgs {
 
 // One warp, one stream.  The packed candidates and the walk-ahead results may have been produced
 // by other SMs moments ago, so they are read past L1 (ld.cg).
-template <int kMode>
+// kAfterGrid: the kernel was launched as a programmatic dependent of the argmax kernel - everything that
+// does not depend on that kernel's output is loaded first, then the warp waits for it to finish.
+template <int kMode, bool kAfterGrid = false>
 __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const AcceptArgs& p, int b, int lane) {
     const int K = p.K;
     const int K1 = K + 1;
@@ -535,6 +539,8 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         if (s != 0) r = load_rec(sam, s);
     }
     const int nd = (p.flags & kNoSpeculation) ? 0 : max(0, min(p.n_draft[b], K));
+    const int d = (lane < K) ? p.drafts[static_cast<long long>(b) * K + lane] : -1;
+    if (kAfterGrid) asm volatile("griddepcontrol.wait;" ::: "memory");
     RecRegs rj = root_rec();     // kTailResume: lane j fetches the record of the state reached after j + 1 drafts
     if (kMode == kTailResume && lane < nd) {
         ps = __ldcg(p.pre_state + static_cast<long long>(b) * K + lane);
@@ -559,7 +565,6 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         }
     }
 
-    const int d = (lane < K) ? p.drafts[static_cast<long long>(b) * K + lane] : -1;
     const unsigned mism = __ballot_sync(kFull, lane < nd && d != am[0]);
     const int a = mism ? (__ffs(mism) - 1) : nd;        // accepted draft tokens
     const int bonus_lo = __shfl_sync(kFull, am[0], a & 31);
@@ -622,7 +627,7 @@ accept_kernel(DeviceSam sam, AcceptArgs p) {
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= p.B) return;
-    accept_stream<kMode>(sam, p, b, lane);
+    accept_stream<kMode, true>(sam, p, b, lane);
 }
 
 }  // namespace samb200
