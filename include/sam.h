@@ -274,7 +274,7 @@ int sam_step_host(const sam_index* idx,
  *
  * sam_build_growing builds the automaton of corpus[0..n) (n may be 0) like sam_build, keeps the
  * builder alive in a thread of its own, and sizes the device blob (sam_sizes) for up to max_tokens
- * tokens: room for 2*max_tokens+2 state records, 6*max_tokens wide edges, a dense root table for token ids
+ * tokens: room for 2*max_tokens+2 state records, 8*max_tokens wide edges, a dense root table for token ids
  * 0..max_token_id, the text, and an 8 MiB staging area for updates.  sam_upload, sam_draft,
  * sam_verify, sam_step, sam_export, sam_sizes and sam_free work as for any other index.
  *   max_tokens    1 .. 2^29, >= n;  max_token_id  largest token id that will ever be indexed

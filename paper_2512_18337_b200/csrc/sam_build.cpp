@@ -62,8 +62,9 @@ int build_index(const int32_t* corpus, int64_t n, const int32_t* seps, int32_t n
         int64_t wide = 0;
         for (int64_t s = 1; s < S; ++s) {
             const int64_t d = out->row_ptr[s + 1] - out->row_ptr[s];
-            if (d >= 3) wide += d;
+            if (d >= 3) wide += (d <= kSortedRowMax) ? d : (int64_t(1) << hash_log2cap(static_cast<int32_t>(d), 2));
         }
+        if (wide >= (int64_t(1) << 31) - 64) return SAM_ERR_TOO_LARGE;   // row offsets are 32-bit
         L.n_wide_edges = wide;
         int64_t span = 0;  // dense root table covers token ids [0, span)
         for (int64_t k = out->row_ptr[0]; k < out->row_ptr[1]; ++k)
@@ -99,9 +100,22 @@ void pack_records(const sam_index& idx, StateRec* rec, Edge* wide, int32_t* root
             r.e[0] = idx.edge_tok[lo];
             r.e[1] = idx.edge_dst[lo];
             if (d == 2) { r.e[2] = idx.edge_tok[lo + 1]; r.e[3] = idx.edge_dst[lo + 1]; }
-        } else if (d >= 3) {
+        } else if (d >= 3 && d <= kSortedRowMax) {
             r.e[0] = static_cast<int32_t>(w);
             for (int64_t k = lo; k < hi; ++k, ++w) { wide[w].tok = idx.edge_tok[k]; wide[w].dst = idx.edge_dst[k]; }
+        } else if (d > kSortedRowMax) {
+            const int32_t lc = hash_log2cap(static_cast<int32_t>(d), 2);
+            const int64_t cap = int64_t(1) << lc;
+            Edge* row = wide + w;
+            for (int64_t k = 0; k < cap; ++k) row[k] = Edge{-1, -1};
+            for (int64_t k = lo; k < hi; ++k) {
+                uint32_t at = hash_slot(idx.edge_tok[k], lc);
+                while (row[at].tok >= 0) at = (at + 1) & static_cast<uint32_t>(cap - 1);
+                row[at] = Edge{idx.edge_tok[k], idx.edge_dst[k]};
+            }
+            r.e[0] = static_cast<int32_t>(w);
+            r.e[1] = lc;
+            w += cap;
         }
         rec[s] = r;
     }

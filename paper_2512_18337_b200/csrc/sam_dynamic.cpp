@@ -34,6 +34,7 @@ struct DynIndex {
     std::vector<int32_t> packed_deg;           // per state: transitions its wide row held when it was last packed
     std::vector<Edge> mirror;                  // host copy of the device's wide array (rows sorted by token)
     int64_t w_used = 0;
+    int64_t compact_every = 0, updates_packed = 0;   // test knob: lay the wide rows out afresh at every k-th update
 
     std::thread worker;
     std::mutex mu;
@@ -53,21 +54,50 @@ int32_t pow2_at_least(int32_t d) {
     return c;
 }
 
-// Record of state s (not the root).  A wide row lives, sorted, in the host mirror of the device's wide
-// array: a row that is new or has outgrown its slot is sorted and placed afresh; otherwise the
-// transitions added since the last packing (the newest nodes of the state's chain) are merged in and
-// redirected ones patched, so that a hub row with thousands of entries is never sorted again.
-// *first / *count tell which part of the row differs from what the device holds.
+// Appends "edges [first, first + count) of the row at `off` changed" to the delta (nothing when segs is null).
+void note_segment(DynIndex& D, Delta* out, int64_t off, int64_t first, int64_t count) {
+    if (!out || count <= 0) return;
+    WideSeg g;
+    g.dst_off = off + first;
+    g.src_off = static_cast<int64_t>(out->seg_edges.size());
+    g.len = static_cast<int32_t>(count);
+    out->segs.push_back(g);
+    const Edge* row = D.mirror.data() + off + first;
+    out->seg_edges.insert(out->seg_edges.end(), row, row + count);
+}
+
+bool place_row(DynIndex& D, int32_t s, int32_t cap) {
+    if (D.w_used + cap > D.w_cap) return false;
+    D.wide_off[s] = static_cast<int32_t>(D.w_used);
+    D.wide_cap[s] = cap;
+    D.w_used += cap;
+    if (D.mirror.size() < static_cast<size_t>(D.w_used)) D.mirror.resize(static_cast<size_t>(D.w_used), Edge{-1, -1});
+    return true;
+}
+
+// Slot of token tok in the hash row (its own slot, or the empty one where it would go).
+uint32_t hash_find(const Edge* row, int32_t lc, int32_t tok) {
+    const uint32_t mask = (1u << lc) - 1u;
+    uint32_t at = hash_slot(tok, lc);
+    while (row[at].tok >= 0 && row[at].tok != tok) at = (at + 1) & mask;
+    return at;
+}
+
+// Record of state s (not the root).  Wide rows live in the host mirror of the device's wide array.
+// Up to kSortedRowMax transitions a row is a sorted array in a power-of-two slot: the transitions added
+// since the last packing (the newest nodes of the state's chain) are merged in, redirected ones patched.
+// Beyond that it is a hash table: a new transition is one slot written, a redirected one one slot
+// patched; the table moves (and is sent whole) only when it is half full.  What differs from the device's
+// copy is appended to `out` (null: nothing is recorded, the caller sends everything).
 // Returns false when the wide area is exhausted.
 bool pack_state(DynIndex& D, int32_t s, StateRec* r, const std::pair<int32_t, int32_t>* redir, size_t n_redir,
-                std::vector<std::pair<int32_t, int32_t>>& tmp, int64_t* first, int64_t* count) {
+                std::vector<std::pair<int32_t, int32_t>>& tmp, Delta* out) {
     const Builder& b = D.b;
     r->len = b.len[s];
     r->link = b.link[s];
     r->firstpos = b.fpos[s];
     r->deg = b.deg[s];
     r->e[0] = r->e[1] = r->e[2] = r->e[3] = -1;
-    *first = *count = 0;
     const int32_t d = b.deg[s];
     if (d <= 2) {
         if (d >= 1) {
@@ -83,54 +113,82 @@ bool pack_state(DynIndex& D, int32_t s, StateRec* r, const std::pair<int32_t, in
         D.wide_cap.resize(b.len.size(), 0);
         D.packed_deg.resize(b.len.size(), 0);
     }
-    if (D.wide_cap[s] < d) {
-        // new slot, whole row
-        const int32_t cap = pow2_at_least(d);
-        if (D.w_used + cap > D.w_cap) return false;
-        D.wide_off[s] = static_cast<int32_t>(D.w_used);
-        D.wide_cap[s] = cap;
-        D.w_used += cap;
-        if (D.mirror.size() < static_cast<size_t>(D.w_used)) D.mirror.resize(static_cast<size_t>(D.w_used), Edge{-1, -1});
-        b.sorted_row(s, tmp);
-        Edge* row = D.mirror.data() + D.wide_off[s];
-        for (int32_t k = 0; k < d; ++k) row[k] = Edge{tmp[k].first, tmp[k].second};
-        *first = 0;
-        *count = d;
-    } else {
-        Edge* row = D.mirror.data() + D.wide_off[s];
-        const int32_t old = D.packed_deg[s];
-        int64_t lowest = d;                                   // lowest position written
-        const int32_t k_new = d - old;
-        if (k_new > 0) {
-            tmp.clear();
-            int32_t x = b.head[s];
-            for (int32_t k = 0; k < k_new; ++k, x = b.e_next[x]) tmp.emplace_back(b.e_tok[x], b.e_dst[x]);
-            std::sort(tmp.begin(), tmp.end());
-            int32_t i = old - 1, j = k_new - 1, w = d - 1;
-            while (j >= 0) {
-                if (i >= 0 && row[i].tok > tmp[j].first) row[w--] = row[i--];
-                else { row[w] = Edge{tmp[j].first, tmp[j].second}; --w; --j; }
+    const int32_t old = D.packed_deg[s];
+    const bool was_hash = D.wide_cap[s] > kSortedRowMax;
+    if (d <= kSortedRowMax) {
+        if (D.wide_cap[s] < d) {
+            // new slot, whole row
+            if (!place_row(D, s, pow2_at_least(d))) return false;
+            b.sorted_row(s, tmp);
+            Edge* row = D.mirror.data() + D.wide_off[s];
+            for (int32_t k = 0; k < d; ++k) row[k] = Edge{tmp[k].first, tmp[k].second};
+            note_segment(D, out, D.wide_off[s], 0, d);
+        } else {
+            Edge* row = D.mirror.data() + D.wide_off[s];
+            int64_t lowest = d;                                   // lowest position written
+            const int32_t k_new = d - old;
+            if (k_new > 0) {
+                tmp.clear();
+                int32_t x = b.head[s];
+                for (int32_t k = 0; k < k_new; ++k, x = b.e_next[x]) tmp.emplace_back(b.e_tok[x], b.e_dst[x]);
+                std::sort(tmp.begin(), tmp.end());
+                int32_t i = old - 1, j = k_new - 1, w = d - 1;
+                while (j >= 0) {
+                    if (i >= 0 && row[i].tok > tmp[j].first) row[w--] = row[i--];
+                    else { row[w] = Edge{tmp[j].first, tmp[j].second}; --w; --j; }
+                }
+                lowest = w + 1;
             }
-            lowest = w + 1;
+            for (size_t q = 0; q < n_redir; ++q) {
+                const int32_t tok = redir[q].second;
+                int32_t lo = 0, hi = d;
+                while (lo < hi) {
+                    const int32_t mid = (lo + hi) >> 1;
+                    if (row[mid].tok < tok) lo = mid + 1; else hi = mid;
+                }
+                if (lo < d && row[lo].tok == tok) {
+                    const int32_t e = b.find(s, tok);
+                    if (e >= 0) row[lo].dst = b.e_dst[e];
+                    if (lo < lowest) lowest = lo;
+                }
+            }
+            note_segment(D, out, D.wide_off[s], lowest, d - lowest);
+        }
+    } else if (!was_hash || 2 * static_cast<int64_t>(d) > D.wide_cap[s]) {
+        // a fresh hash table (the row was a sorted array so far, or the table is half full), sent whole
+        const int32_t lc = hash_log2cap(d, 4);
+        if (!place_row(D, s, 1 << lc)) return false;
+        Edge* row = D.mirror.data() + D.wide_off[s];
+        for (int32_t k = 0; k < (1 << lc); ++k) row[k] = Edge{-1, -1};
+        for (int32_t x = b.head[s]; x >= 0; x = b.e_next[x]) row[hash_find(row, lc, b.e_tok[x])] = Edge{b.e_tok[x], b.e_dst[x]};
+        note_segment(D, out, D.wide_off[s], 0, int64_t(1) << lc);
+    } else {
+        int32_t lc = 0;
+        while ((1 << lc) < D.wide_cap[s]) ++lc;
+        Edge* row = D.mirror.data() + D.wide_off[s];
+        int32_t x = b.head[s];
+        for (int32_t k = 0; k < d - old; ++k, x = b.e_next[x]) {          // the transitions added since the last packing
+            const uint32_t at = hash_find(row, lc, b.e_tok[x]);
+            row[at] = Edge{b.e_tok[x], b.e_dst[x]};
+            note_segment(D, out, D.wide_off[s], at, 1);
         }
         for (size_t q = 0; q < n_redir; ++q) {
             const int32_t tok = redir[q].second;
-            int32_t lo = 0, hi = d;
-            while (lo < hi) {
-                const int32_t mid = (lo + hi) >> 1;
-                if (row[mid].tok < tok) lo = mid + 1; else hi = mid;
-            }
-            if (lo < d && row[lo].tok == tok) {
-                const int32_t e = b.find(s, tok);
-                if (e >= 0) row[lo].dst = b.e_dst[e];
-                if (lo < lowest) lowest = lo;
+            const uint32_t at = hash_find(row, lc, tok);
+            const int32_t e = b.find(s, tok);
+            if (row[at].tok == tok && e >= 0 && row[at].dst != b.e_dst[e]) {
+                row[at].dst = b.e_dst[e];
+                note_segment(D, out, D.wide_off[s], at, 1);
             }
         }
-        *first = lowest;
-        *count = d - lowest;
     }
     D.packed_deg[s] = d;
     r->e[0] = D.wide_off[s];
+    if (D.wide_cap[s] > kSortedRowMax) {
+        int32_t lc = 0;
+        while ((1 << lc) < D.wide_cap[s]) ++lc;
+        r->e[1] = lc;
+    }
     return true;
 }
 
@@ -148,8 +206,7 @@ int pack_full(DynIndex& D, Delta* out) {
     D.w_used = 0;
     std::vector<std::pair<int32_t, int32_t>> tmp;
     for (int64_t s = 1; s < S; ++s) {
-        int64_t first = 0, count = 0;
-        if (!pack_state(D, static_cast<int32_t>(s), &out->all_rec[s], nullptr, 0, tmp, &first, &count)) return SAM_ERR_TOO_LARGE;
+        if (!pack_state(D, static_cast<int32_t>(s), &out->all_rec[s], nullptr, 0, tmp, nullptr)) return SAM_ERR_TOO_LARGE;
     }
     out->all_wide.assign(D.mirror.begin(), D.mirror.begin() + D.w_used);
     StateRec& r0 = out->all_rec[0];
@@ -169,12 +226,17 @@ int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
     out->rec_ids.reserve(b.dirty.size());
     out->recs.reserve(b.dirty.size());
     std::sort(b.redirected.begin(), b.redirected.end());
+    if (D.compact_every > 0 && ++D.updates_packed % D.compact_every == 0) {
+        Delta fresh;
+        const int rc = pack_full(D, &fresh);
+        *out = std::move(fresh);
+        return rc;
+    }
     for (int32_t s : b.dirty) {
         StateRec r;
         const auto lo = std::lower_bound(b.redirected.begin(), b.redirected.end(), std::make_pair(s, INT32_MIN));
         const auto hi = std::lower_bound(lo, b.redirected.end(), std::make_pair(s + 1, INT32_MIN));
-        int64_t first = 0, count = 0;
-        if (!pack_state(D, s, &r, lo == hi ? nullptr : &*lo, static_cast<size_t>(hi - lo), tmp, &first, &count)) {
+        if (!pack_state(D, s, &r, lo == hi ? nullptr : &*lo, static_cast<size_t>(hi - lo), tmp, out)) {
             // wide area exhausted: lay everything out afresh and send the whole image instead
             Delta fresh;
             const int rc = pack_full(D, &fresh);
@@ -183,15 +245,6 @@ int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
         }
         out->rec_ids.push_back(s);
         out->recs.push_back(r);
-        if (count > 0) {
-            WideSeg g;
-            g.dst_off = D.wide_off[s] + first;
-            g.src_off = static_cast<int64_t>(out->seg_edges.size());
-            g.len = static_cast<int32_t>(count);
-            out->segs.push_back(g);
-            const Edge* row = D.mirror.data() + D.wide_off[s] + first;
-            out->seg_edges.insert(out->seg_edges.end(), row, row + count);
-        }
     }
     // root: the last change of a token wins
     std::unordered_map<int32_t, int32_t> last;
@@ -256,9 +309,11 @@ int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tok
         D = new DynIndex();
         D->max_tokens = max_tokens;
         D->s_cap = 2 * max_tokens + 2;
-        // rows hold at most 3N transitions in total and a row's slot is less than twice its length, so a fresh
-        // layout always fits 6N; the rest of the area absorbs rows that outgrew their slot
-        double per_token = 6.0;
+        // sorted rows sit in power-of-two slots (less than twice their length), hash rows are between an eighth
+        // and a half full; 8 edges of room per token leaves ample slack for the corpora this is meant for, and
+        // when the area does fill up the rows are laid out afresh (SAM_ERR_TOO_LARGE if even that does not fit)
+        if (const char* e = std::getenv("SAM_B200_COMPACT_EVERY")) D->compact_every = std::atoll(e);   // test knob
+        double per_token = 8.0;
         if (const char* e = std::getenv("SAM_B200_WIDE_EDGES_PER_TOKEN")) {   // tuning / test knob
             const double v = std::atof(e);
             if (v >= 0.25 && v <= 64.0) per_token = v;

@@ -10,7 +10,13 @@ namespace samb200 {
 // One 32-byte record per state = one DRAM/L2 sector per state visit.
 //   deg == 1 : e[0]=tok0 e[1]=dst0                      (transition stored inline)
 //   deg == 2 : e[0]=tok0 e[1]=dst0 e[2]=tok1 e[3]=dst1  (both inline, ascending)
-//   deg >= 3 : e[0]=offset of the state's row in the wide-edge array (units of one edge)
+//   3 <= deg <= kSortedRowMax : e[0]=offset of the state's row in the wide-edge array (units of one
+//              edge), e[1] = -1; the row holds the deg transitions ascending by token - one warp-wide
+//              read finds any of them
+//   deg > kSortedRowMax : e[0]=offset, e[1]=log2 of the row's capacity; the row is an open-addressing
+//              hash table (linear probing from hash_slot(tok), empty slots have tok = -1, never more
+//              than half full, nothing is ever deleted) - one warp-wide read of 32 consecutive slots
+//              finds a transition or proves its absence in all but freak cases
 //   root     : transitions come from the dense root table, e[] unused
 struct StateRec {
     int32_t len, link, firstpos, deg;
@@ -18,7 +24,27 @@ struct StateRec {
 };
 static_assert(sizeof(StateRec) == 32, "one sector per state");
 
-struct Edge { int32_t tok, dst; };  // wide rows: ascending by tok
+struct Edge { int32_t tok, dst; };
+
+constexpr int32_t kSortedRowMax = 32;
+
+#ifdef __CUDACC__
+#define SAM_HD __host__ __device__ __forceinline__
+#else
+#define SAM_HD inline
+#endif
+// First slot probed for token tok in a hash row of 2^log2cap slots (multiplicative hashing).
+SAM_HD uint32_t hash_slot(int32_t tok, int32_t log2cap) {
+    return (static_cast<uint32_t>(tok) * 0x9E3779B1u) >> (32 - log2cap);
+}
+// Capacity (log2) of a fresh hash row for deg transitions: the smallest power of two >= room * deg
+// (room = 2 for an index that never grows; 4 for one that does, so that a row can double its population
+// before it has to move).
+SAM_HD int32_t hash_log2cap(int32_t deg, int32_t room) {
+    int32_t l = 7;
+    while ((int64_t(1) << l) < int64_t(room) * deg) ++l;
+    return l;
+}
 
 // Where things sit inside the caller's device blob (byte offsets, 256-byte aligned).
 // A growing index sizes every section for its capacity and adds a staging area for updates.

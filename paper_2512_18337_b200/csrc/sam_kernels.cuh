@@ -36,29 +36,29 @@ __device__ __forceinline__ RecRegs root_rec() {
     return r;
 }
 
-// Warp-cooperative search of one ascending row of `deg` (tok, dst) pairs: 32-way narrowing
-// until at most 32 candidates remain, then one pass in which every lane compares its own entry.
-// Each round is one dependent memory access.
-__device__ __forceinline__ int row_search(const Edge* __restrict__ row, int deg, int c, int lane) {
-    int lo = 0, hi = deg;
-    while (hi - lo > 32) {
-        const int step = (hi - lo + 31) >> 5;
-        const int i = lo + lane * step;
-        const bool in = i < hi;
-        const int t = in ? __ldg(&row[i].tok) : 0;
-        const unsigned le = __ballot_sync(kFull, in && t <= c);
-        if (le == 0) return -1;             // c is below the first pivot of the range
-        const int k = __popc(le) - 1;       // pivots ascend, so `le` is a prefix mask
-        lo = lo + k * step;
-        hi = min(lo + step, hi);
-    }
-    const int i = lo + lane;
+// One warp-wide read of an ascending row of at most 32 (tok, dst) pairs.
+__device__ __forceinline__ int sorted_row_lookup(const Edge* __restrict__ row, int deg, int c, int lane) {
     int2 e = make_int2(0, -1);
-    const bool in = i < hi;
-    if (in) e = __ldg(reinterpret_cast<const int2*>(row + i));
+    const bool in = lane < deg;
+    if (in) e = __ldg(reinterpret_cast<const int2*>(row + lane));
     const unsigned hit = __ballot_sync(kFull, in && e.x == c);
     if (hit == 0) return -1;
     return __shfl_sync(kFull, e.y, __ffs(hit) - 1);
+}
+
+// Hash row: 32 consecutive slots from the token's home slot per round.  Insertion took the first empty
+// slot from there and nothing is ever deleted, so a token that is present sits before the first empty slot.
+__device__ __forceinline__ int hash_row_lookup(const Edge* __restrict__ row, int log2cap, int c, int lane) {
+    if (c < 0) return -1;
+    const unsigned mask = (1u << log2cap) - 1u;
+    const unsigned home = hash_slot(c, log2cap);
+    for (unsigned w = 0; w <= mask; w += 32) {
+        const int2 e = __ldg(reinterpret_cast<const int2*>(row + ((home + w + lane) & mask)));
+        const unsigned hit = __ballot_sync(kFull, e.x == c);
+        if (hit != 0) return __shfl_sync(kFull, e.y, __ffs(hit) - 1);
+        if (__ballot_sync(kFull, e.x < 0) != 0) return -1;
+    }
+    return -1;
 }
 
 // Destination of the transition (s, c) or -1. `r` is the record of s.
@@ -72,7 +72,8 @@ __device__ __forceinline__ int transition(const DeviceSam& sam, int s, const Rec
         if (deg == 2 && r.b.z == c) return r.b.w;
         return -1;
     }
-    return row_search(sam.wide + r.b.x, deg, c, lane);
+    if (deg <= kSortedRowMax) return sorted_row_lookup(sam.wide + r.b.x, deg, c, lane);
+    return hash_row_lookup(sam.wide + r.b.x, r.b.y, c, lane);
 }
 
 // Consume one token: a transition extends the match by one; on a miss follow the suffix link

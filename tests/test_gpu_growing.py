@@ -42,15 +42,15 @@ def _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm):
     return d_o, nd_o
 
 
-@pytest.mark.parametrize("seed,wide_per_token", [(0, None), (1, "0.8")])
-def test_draft_parity_while_the_text_grows(seed, wide_per_token, monkeypatch):
-    """With one wide edge of room per token (a tuning knob of the library) the wide rows run out of room
-    along the way and are laid out afresh (whole-image updates); the default keeps every update incremental."""
+@pytest.mark.parametrize("seed,compact_every", [(0, None), (1, "4")])
+def test_draft_parity_while_the_text_grows(seed, compact_every, monkeypatch):
+    """With the library's test knob set, every fourth update lays the wide rows out afresh and is sent as a whole
+    image (what happens by itself when the wide area fills up); the default keeps every update incremental."""
     rng = np.random.default_rng(seed)
     sep, K, mm, B, ld = 1000, 6, 2, 48, 12
     text = _hub_text(rng, 3000, sep)
-    if wide_per_token is not None:
-        monkeypatch.setenv("SAM_B200_WIDE_EDGES_PER_TOKEN", wide_per_token)
+    if compact_every is not None:
+        monkeypatch.setenv("SAM_B200_COMPACT_EVERY", compact_every)
     index = S.SamIndex(text, [sep], max_tokens=12000, max_token_id=sep + 50)
     osam = oracle.OracleSAM(text, [sep])
     st = torch.zeros(B, dtype=torch.int32, device=DEV)
@@ -88,7 +88,7 @@ def test_draft_parity_while_the_text_grows(seed, wide_per_token, monkeypatch):
     assert moved > 0
     inc, full, nbytes = S.sam_update_stats(index.handle)
     assert inc + full == 14 and nbytes > 0
-    assert (full > 0) == (wide_per_token is not None)
+    assert full == (3 if compact_every is not None else 0)
     ex, oe = S.sam_export(index.handle), osam.export()
     for k in oe:
         assert (ex[k] == oe[k]).all(), k
