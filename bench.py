@@ -154,7 +154,7 @@ def run_ours(args):
     base = W.CONFIGS[args.config]
     # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
     # read-only automaton is replicated; no data-path collective
-    cfg = base.scaled(steps=args.warmup + args.steps + args.split_steps + args.e2e_steps + 1)
+    cfg = base.scaled(steps=args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1)
     stream_cfg = cfg.scaled(seed=cfg.seed + 7919 * rank) if rank > 0 else cfg
 
     t0 = time.time()
@@ -279,30 +279,45 @@ def run_ours(args):
         torch.cuda.synchronize()
         sb = S.sam_step_host_staging_bytes(V, B, K, V)
         staging = torch.empty(sb, dtype=torch.uint8, device=device)
-        e2e_tokens, e2e_s = 0, 0.0
-        for i in range(args.e2e_steps):
-            t = args.warmup + args.steps + i
-            ow = feeder.overwrites(t, h["drafts"].numpy(), h["n_draft"].numpy())
-            saved = hraw[ow["row"], ow["col"]].copy()
-            hraw[ow["row"], ow["col"]] = ow["bits"]
-            torch.cuda.synchronize()
-            c0 = time.perf_counter()
-            S.sam_step_host(index.handle, host_logits, V, B, K, V, h["drafts"], h["n_draft"], h["argmax"],
-                            h["accepted"], h["n_accepted"], h["state"], h["mlen"], cfg.min_match,
-                            h["drafts"], h["n_draft"], staging, sb)
-            c1 = time.perf_counter()
-            hraw[ow["row"], ow["col"]] = saved
-            n_acc = h["n_accepted"].numpy().copy()
-            feeder.advance(n_acc)
-            if i > 0 or args.e2e_steps == 1:       # first host step warms the pinned path
-                e2e_tokens += int(n_acc.sum())
-                e2e_s += c1 - c0
-        h2d = logits.numel() * 2 + (B * K + 3 * B) * 4
+        def host_loop(flags, t_base):
+            toks, secs, rows = 0, 0.0, 0
+            for i in range(args.e2e_steps):
+                t = t_base + i
+                ow = feeder.overwrites(t, h["drafts"].numpy(), h["n_draft"].numpy())
+                saved = hraw[ow["row"], ow["col"]].copy()
+                hraw[ow["row"], ow["col"]] = ow["bits"]
+                used_rows = int(np.clip(h["n_draft"].numpy(), 0, K).sum()) + B
+                torch.cuda.synchronize()
+                c0 = time.perf_counter()
+                S.sam_step_host_ex(index.handle, host_logits, V, B, K, V, h["drafts"], h["n_draft"], h["argmax"],
+                                   h["accepted"], h["n_accepted"], h["state"], h["mlen"], cfg.min_match,
+                                   h["drafts"], h["n_draft"], flags, staging, sb)
+                c1 = time.perf_counter()
+                hraw[ow["row"], ow["col"]] = saved
+                n_acc = h["n_accepted"].numpy().copy()
+                feeder.advance(n_acc)
+                if i > 0 or args.e2e_steps == 1:       # first host step warms the pinned path
+                    toks += int(n_acc.sum())
+                    secs += c1 - c0
+                    rows += used_rows
+            return toks, secs, rows
+
+        t_e2e = args.warmup + args.steps + args.split_steps
+        e2e_tokens, e2e_s, _ = host_loop(0, t_e2e)
+        skip_tokens, skip_s, skip_rows = host_loop(S.SAM_STEP_SKIP_UNUSED_ROWS, t_e2e + args.e2e_steps)
+        n_timed = max(1, args.e2e_steps - 1)
+        small = (B * K + 3 * B) * 4
+        h2d = logits.numel() * 2 + small
         d2h = (2 * B * (K + 1) + B * K + 4 * B) * 4
         e2e_tokens, e2e_ms = reduce_over_ranks(e2e_tokens, e2e_s * 1e3, world, device)
+        skip_tokens, skip_ms = reduce_over_ranks(skip_tokens, skip_s * 1e3, world, device)
         e2e = {"value": e2e_tokens / (e2e_ms / 1e3) if e2e_ms > 0 else None, "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "steps": max(1, args.e2e_steps - 1), "api": "sam_step_host (pinned host buffers, wall clock incl. sync)"}
+               "steps": n_timed, "api": "sam_step_host (pinned host buffers, wall clock incl. sync)",
+               "skip_unused_rows": {"value": skip_tokens / (skip_ms / 1e3) if skip_ms > 0 else None, "unit": UNIT,
+                                    "h2d_bytes_per_step": skip_rows / n_timed * V * 2 + small,
+                                    "api": "sam_step_host_ex with SAM_STEP_SKIP_UNUSED_ROWS: only rows 0..n_draft[b] "
+                                           "cross the bus (a different contract: the other rows are not arg-maxed)"}}
         del staging, host_logits
 
     all_tokens, max_ms = reduce_over_ranks(tokens, total_ms, world, device)
@@ -357,7 +372,11 @@ def run_ours(args):
         "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
                      "traffic": (NCU_DRAM_BYTES_PER_ROW * (rows_read_per_step if args.skip_unused_rows else R)) if NCU_DRAM_BYTES_PER_ROW else None,
-                     "algorithmic_bytes": alg_bytes},
+                     "algorithmic_bytes": alg_bytes,
+                     "whole_step": {"ms": total_ms / args.steps, "achieved": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9,
+                                    "frac": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9 / peak,
+                                    "note": "the same bytes over the event bracket of the whole step in the timed region "
+                                            "(argmax + accept + walk + draft)"}},
         "walk": walk,
         "ote": st["ote"], "shr": st["shr"], "mean_n_draft": st["mean_n_draft"],
         "device_counters": {"passes": dev_counters[0], "committed": dev_counters[1], "proposed": dev_counters[2],

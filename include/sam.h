@@ -265,6 +265,17 @@ int sam_step_host(const sam_index* idx,
                   int32_t* next_drafts, int32_t* next_n_draft,
                   void* staging, int64_t staging_bytes, void* cuda_stream);
 
+/* sam_step_host with step options (SAM_STEP_*).  With SAM_STEP_SKIP_UNUSED_ROWS only rows 0..n_draft[b]
+ * of every stream are copied to the device (one copy per stream) - the host-to-device traffic, which
+ * dominates this call, shrinks with the proposals. */
+int sam_step_host_ex(const sam_index* idx,
+                     const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                     const int32_t* drafts, const int32_t* n_draft,
+                     int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                     int32_t* state, int32_t* matched_len, int32_t min_match,
+                     int32_t* next_drafts, int32_t* next_n_draft, uint32_t flags,
+                     void* staging, int64_t staging_bytes, void* cuda_stream);
+
 /* ---------------------------------------------------------------- growing index */
 
 /* An index that keeps absorbing text after it was built (Section 5.4.2: verified tokens are

@@ -52,6 +52,8 @@ _SIGNATURES = {
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
+    "sam_step_host_ex": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                                   _vp, _vp, _i32, _vp, _vp, C.c_uint32, _vp, _i64, _vp]),
     "sam_workspace_status": (C.c_int, [_vp, _i32, _i32, C.POINTER(_i32), _vp]),
     "sam_set_argmax_variant": (C.c_int, [_i32]),
     "sam_profile_enable": (C.c_int, [_i32]),
@@ -367,6 +369,15 @@ def sam_step_host(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_o
                                  _hostptr(argmax_out), _hostptr(accepted), _hostptr(n_accepted), _hostptr(state),
                                  _hostptr(matched_len), min_match, _hostptr(next_drafts), _hostptr(next_n_draft),
                                  _dev(staging), staging_bytes, _stream(stream)), "sam_step_host")
+
+
+def sam_step_host_ex(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                     state, matched_len, min_match, next_drafts, next_n_draft, flags, staging, staging_bytes, stream=None):
+    """sam_step_host with step options; with SAM_STEP_SKIP_UNUSED_ROWS only the used rows are copied."""
+    _check(_load().sam_step_host_ex(handle, _hostptr(logits), row_stride, B, K, V, _hostptr(drafts), _hostptr(n_draft),
+                                    _hostptr(argmax_out), _hostptr(accepted), _hostptr(n_accepted), _hostptr(state),
+                                    _hostptr(matched_len), min_match, _hostptr(next_drafts), _hostptr(next_n_draft),
+                                    flags, _dev(staging), staging_bytes, _stream(stream)), "sam_step_host_ex")
 
 
 def sam_workspace_status(workspace, B: int, K: int, stream=None) -> int:

@@ -760,7 +760,19 @@ int sam_step_host(const sam_index* idx,
                   int32_t* state, int32_t* matched_len, int32_t min_match,
                   int32_t* next_drafts, int32_t* next_n_draft,
                   void* staging, int64_t staging_bytes, void* cuda_stream) {
+    return sam_step_host_ex(idx, logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                            state, matched_len, min_match, next_drafts, next_n_draft, 0, staging, staging_bytes, cuda_stream);
+}
+
+int sam_step_host_ex(const sam_index* idx,
+                     const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                     const int32_t* drafts, const int32_t* n_draft,
+                     int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                     int32_t* state, int32_t* matched_len, int32_t min_match,
+                     int32_t* next_drafts, int32_t* next_n_draft, uint32_t flags,
+                     void* staging, int64_t staging_bytes, void* cuda_stream) {
     HostStepLayout L;
+    if (flags & ~static_cast<uint32_t>(SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS)) return SAM_ERR_INVALID_ARG;
     if (!idx || !host_step_layout(row_stride_elems, B, K, V, &L) || min_match < 1) return SAM_ERR_INVALID_ARG;
     if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
     if (B == 0) return SAM_OK;
@@ -771,7 +783,19 @@ int sam_step_host(const sam_index* idx,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* d = static_cast<char*>(staging);
     const size_t bB = static_cast<size_t>(B) * 4, bK = bB * K, bR = bB * (K + 1);
-    SAM_CUDA(cudaMemcpyAsync(d + L.logits, logits_bf16, static_cast<size_t>(L.logits_bytes), cudaMemcpyHostToDevice, st));
+    if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
+        // only the rows the step will read cross the bus: rows 0..n_draft[b] of every stream, one copy per stream
+        const char* src = static_cast<const char*>(logits_bf16);
+        for (int32_t b = 0; b < B; ++b) {
+            int32_t nd = (flags & SAM_STEP_NO_SPECULATION) ? 0 : n_draft[b];
+            nd = nd < 0 ? 0 : (nd > K ? K : nd);
+            const int64_t first = static_cast<int64_t>(b) * (K + 1) * row_stride_elems * 2;
+            const int64_t bytes = (static_cast<int64_t>(nd) * row_stride_elems + V) * 2;
+            SAM_CUDA(cudaMemcpyAsync(d + L.logits + first, src + first, static_cast<size_t>(bytes), cudaMemcpyHostToDevice, st));
+        }
+    } else {
+        SAM_CUDA(cudaMemcpyAsync(d + L.logits, logits_bf16, static_cast<size_t>(L.logits_bytes), cudaMemcpyHostToDevice, st));
+    }
     SAM_CUDA(cudaMemcpyAsync(d + L.drafts, drafts, bK, cudaMemcpyHostToDevice, st));
     SAM_CUDA(cudaMemcpyAsync(d + L.n_draft, n_draft, bB, cudaMemcpyHostToDevice, st));
     SAM_CUDA(cudaMemcpyAsync(d + L.state, state, bB, cudaMemcpyHostToDevice, st));
@@ -779,10 +803,11 @@ int sam_step_host(const sam_index* idx,
     SAM_CUDA(cudaMemsetAsync(d + L.ws, 0, static_cast<size_t>(L.ws_bytes), st));
     int32_t* dd = reinterpret_cast<int32_t*>(d + L.drafts);
     int32_t* dn = reinterpret_cast<int32_t*>(d + L.n_draft);
-    const int rc = sam_step(idx, d + L.logits, row_stride_elems, B, K, V, dd, dn,
-                            reinterpret_cast<int32_t*>(d + L.argmax), reinterpret_cast<int32_t*>(d + L.accepted),
-                            reinterpret_cast<int32_t*>(d + L.n_accepted), reinterpret_cast<int32_t*>(d + L.state),
-                            reinterpret_cast<int32_t*>(d + L.mlen), min_match, dd, dn, d + L.ws, L.ws_bytes, st);
+    const int rc = sam_step_ex(idx, d + L.logits, row_stride_elems, B, K, V, dd, dn,
+                               reinterpret_cast<int32_t*>(d + L.argmax), reinterpret_cast<int32_t*>(d + L.accepted),
+                               reinterpret_cast<int32_t*>(d + L.n_accepted), reinterpret_cast<int32_t*>(d + L.state),
+                               reinterpret_cast<int32_t*>(d + L.mlen), min_match, dd, dn, flags, nullptr,
+                               d + L.ws, L.ws_bytes, st);
     if (rc != SAM_OK) return rc;
     SAM_CUDA(cudaMemcpyAsync(argmax_out, d + L.argmax, bR, cudaMemcpyDeviceToHost, st));
     SAM_CUDA(cudaMemcpyAsync(accepted, d + L.accepted, bR, cudaMemcpyDeviceToHost, st));

@@ -177,3 +177,44 @@ def test_vocabulary_shards_merge_to_the_full_row(shards, multiple):
         f_g.advance(g["n_accepted"])
         f_o.advance(o["n_accepted"])
         dg, ndg, do, ndo = g["drafts"], g["n_draft"], o["drafts"], o["n_draft"]
+
+
+@pytest.mark.parametrize("flags", [0, 2, 3])
+def test_host_buffer_step_with_options(flags):
+    """sam_step_host_ex: everything in host memory; with SAM_STEP_SKIP_UNUSED_ROWS only the used rows are copied
+    to the device, so the staging area is poisoned first to show that nothing else is read."""
+    cfg = W.CONFIGS[0].scaled(B=9, steps=5)
+    c = cfg
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    noise = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+    index = S.SamIndex(corpus, [cfg.separator])
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    f_o = W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = f_o.prime_tokens()
+    do, ndo = cpu.prime(toks, n)
+    h = dict(drafts=do.copy(), n_draft=ndo.copy(), argmax=np.zeros((c.B, c.K + 1), np.int32),
+             accepted=np.zeros((c.B, c.K + 1), np.int32), n_accepted=np.zeros(c.B, np.int32),
+             state=cpu.state.copy(), mlen=cpu.mlen.copy())
+    sb = S.sam_step_host_staging_bytes(c.vocab, c.B, c.K, c.vocab)
+    staging = torch.empty(sb, dtype=torch.uint8, device=DEV)
+    host_bits = noise.copy()
+    for t in range(c.steps):
+        ow = f_o.overwrites(t, do, ndo if not (flags & 1) else np.zeros(c.B, np.int32))
+        keep = np.arange(ow["row"].shape[0])
+        sv = cpu.poke(ow["row"], ow["col"], ow["bits"], keep)
+        sv_h = host_bits[ow["row"], ow["col"]].copy()
+        host_bits[ow["row"], ow["col"]] = ow["bits"]
+        staging.fill_(0x7F)          # 0x7F7F as bf16 is a huge number: a row that was not copied would win every argmax
+        S.sam_step_host_ex(index.handle, host_bits, c.vocab, c.B, c.K, c.vocab, h["drafts"], h["n_draft"], h["argmax"],
+                           h["accepted"], h["n_accepted"], h["state"], h["mlen"], c.min_match,
+                           h["drafts"], h["n_draft"], flags, staging, sb)
+        o = cpu.sam.step_ex(cpu.bits, c.B, c.K, c.vocab, do, ndo, cpu.state, cpu.mlen, c.min_match, flags)
+        cpu.unpoke(ow["row"], ow["col"], sv)
+        host_bits[ow["row"], ow["col"]] = sv_h
+        assert (h["argmax"] == o["argmax"]).all() and (h["accepted"] == o["accepted"]).all(), t
+        assert (h["n_accepted"] == o["n_accepted"]).all() and (h["state"] == cpu.state).all() and (h["mlen"] == cpu.mlen).all()
+        assert (h["drafts"] == o["drafts"]).all() and (h["n_draft"] == o["n_draft"]).all()
+        f_o.advance(o["n_accepted"])
+        do, ndo = o["drafts"], o["n_draft"]
