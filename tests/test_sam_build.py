@@ -156,3 +156,31 @@ def test_growing_index_from_empty_and_limits():
         assert lib.sam_sync(hs, None, None) == -1
     finally:
         S.sam_free(hs)
+
+
+def test_argument_checks_that_need_no_device():
+    """Entry points reject bad sizes, flags and null pointers before they touch CUDA."""
+    lib = S.binding._load()
+    assert S.sam_workspace_bytes(4, 8) % 256 == 0
+    assert S.sam_workspace_bytes(8, 8) > S.sam_workspace_bytes(4, 8) > S.sam_workspace_bytes(4, 1)
+    assert lib.sam_workspace_bytes(-1, 4) == -1 and lib.sam_workspace_bytes(4, 0) == -1 and lib.sam_workspace_bytes(4, 33) == -1
+    assert lib.sam_verify_ex(None, 8, 1, 1, 8, None, None, None, None, None, 8, None, None, 0, None) == -1     # unknown flag
+    assert lib.sam_verify_ex(None, 8, 0, 1, 8, None, None, None, None, None, 0, None, None, 0, None) == 0      # B = 0
+    assert lib.sam_verify_ex(None, 7, 1, 1, 8, None, None, None, None, None, 0, None, None, 0, None) == -1     # stride < V
+    assert lib.sam_step_ex(None, None, 8, 1, 1, 8, None, None, None, None, None, None, None, 1, None, None, 0, None,
+                           None, 0, None) == -1                                                                # no index
+    assert lib.sam_argmax_partial(None, 8, 0, 8, 0, None, None) == 0                                           # no rows
+    assert lib.sam_argmax_partial(None, 8, 1, 8, -1, None, None) == -1                                         # bad offset
+    assert lib.sam_argmax_partial(None, 8, 1, 8, 0, None, None) == -1                                          # null pointers
+    assert lib.sam_set_bytes(0) == -1 and lib.sam_set_bytes(2) % 256 == 0
+    assert lib.sam_adaptive_switch(100, 4, 100, 4) == 1 and lib.sam_adaptive_switch(101, 4, 100, 4) == 0
+    assert lib.sam_adaptive_switch(100, 5, 100, 4) == 0
+    for ctx, bs in [(1, 1), (10 ** 6, 1), (1, 10 ** 4), (32768, 64), (32769, 64), (32768, 65)]:
+        assert bool(lib.sam_adaptive_switch(ctx, bs, 32768, 64)) == oracle.speculation_enabled(ctx, bs, 32768, 64)
+    h = S.sam_build(np.array([1, 2, 3], np.int32), [9])
+    try:   # hot-path calls before sam_upload
+        assert lib.sam_draft(h, 1, None, None, None, 0, None, 2, 1, None, None, None) == -3
+        assert lib.sam_renormalize(h, 1, None, None, None) == -3
+    finally:
+        S.sam_free(h)
+    assert S.sam_strerror(-3).startswith("automaton not uploaded")
