@@ -667,7 +667,7 @@ def run_multi(args):
     st, ml = torch.zeros((B, M), **i32), torch.zeros((B, M), **i32)
     drafts, n_draft, chosen = torch.full((B, K), -1, **i32), torch.zeros(B, **i32), torch.zeros(B, **i32)
     am, acc, nacc = torch.zeros((B, K + 1), **i32), torch.zeros((B, K + 1), **i32), torch.zeros(B, **i32)
-    wsb = S.sam_workspace_bytes(B, K)
+    wsb = S.sam_multi_workspace_bytes(B, K, M)
     ws = torch.empty(wsb, dtype=torch.uint8, device=device)
     S.sam_workspace_init(ws, wsb)
     raw = logits.view(torch.int16)
@@ -688,10 +688,16 @@ def run_multi(args):
             drafted += int(n_draft.sum())
             torch.cuda._sleep(args.presleep_cycles)
             ev[i][0].record()
-        S.sam_verify(logits, V, B, K, V, drafts, n_draft, am, acc, nacc, ws, wsb)
-        if i >= 0:
-            ev[i][1].record()
-        S.sam_multi_draft(sset.handle, B, M, slots, weights, st, ml, acc, K + 1, nacc, K, cfg.min_match, drafts, n_draft, chosen)
+        if args.multi_unfused:
+            S.sam_verify(logits, V, B, K, V, drafts, n_draft, am, acc, nacc, ws, wsb)
+            if i >= 0:
+                ev[i][1].record()
+            S.sam_multi_draft(sset.handle, B, M, slots, weights, st, ml, acc, K + 1, nacc, K, cfg.min_match, drafts, n_draft, chosen)
+        else:
+            if i >= 0:
+                ev[i][1].record()
+            S.sam_multi_step(sset.handle, logits, V, B, K, V, drafts, n_draft, am, acc, nacc, M, slots, weights, st, ml,
+                             cfg.min_match, drafts, n_draft, chosen, ws, wsb)
         if i >= 0:
             ev[i][2].record()
         torch.cuda.synchronize()
@@ -707,8 +713,9 @@ def run_multi(args):
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "dtype": "bf16 compare / int32",
         "data": "synthetic",
         "config": {"workload": cfg.name + f" split into {M} member automata, every stream holds all {M}", "B": B, "K": K,
-                   "V": V, "timing": "CUDA events around sam_verify + sam_multi_draft"},
-        "multi_draft_kernel_ms": ms_multi / args.steps, "slot_walks_per_s": B * M * args.steps / (ms_multi / 1e3),
+                   "V": V, "api": "sam_verify + sam_multi_draft" if args.multi_unfused else "sam_multi_step",
+                   "timing": "CUDA events around the step"},
+        "multi_draft_kernel_ms": (ms_multi / args.steps) if args.multi_unfused else None,
         "mean_n_draft": drafted / (B * args.steps), "ote": tokens / (B * args.steps), "members_build_s": t_build,
     }))
 
@@ -738,6 +745,7 @@ def main():
                          "all shards one after the other on a single GPU); prints a separate JSON line")
     ap.add_argument("--multi", type=int, default=0,
                     help="> 0: closed loop with composite drafting over that many member automata (1..8); separate JSON line")
+    ap.add_argument("--multi-unfused", action="store_true", help="with --multi: sam_verify + sam_multi_draft instead of sam_multi_step")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()

@@ -92,7 +92,7 @@ void sam_free(sam_index* idx);
 int64_t sam_workspace_bytes(int32_t B, int32_t K);
 
 /* Zero-fills the scratch (device, 8-byte aligned) on the stream.  Required once before the
- * first sam_verify / sam_step that uses it; every successful call leaves it zeroed again.
+ * first sam_verify / sam_step that uses it; every successful call leaves it ready for the next one.
  * Call it again after a hot-path call returned an error.  Calls that share one workspace
  * must not overlap on the device. */
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
@@ -363,6 +363,22 @@ int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slo
                     int32_t* state, int32_t* matched_len, const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
                     int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, int32_t* chosen,
                     void* cuda_stream);
+
+/* One decoding step with composite drafting, fused like sam_step: vocabulary argmax over all B*(K+1) rows
+ * (with every slot's walk-ahead over the drafts riding along), accept, then every slot follows the
+ * committed tokens in its own automaton and the slots compete for the next draft - the result is what
+ * sam_verify followed by sam_multi_draft(new_tokens = accepted, n_new = n_accepted) gives.
+ *   workspace   device scratch of sam_multi_workspace_bytes(B, K, M), zeroed once by sam_workspace_init
+ *   other arguments as in sam_verify and sam_multi_draft; next_drafts / next_n_draft may alias drafts / n_draft
+ * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_SMALL, SAM_ERR_CUDA. */
+int64_t sam_multi_workspace_bytes(int32_t B, int32_t K, int32_t M);
+int sam_multi_step(const sam_set* set,
+                   const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                   const int32_t* drafts, const int32_t* n_draft,
+                   int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                   int32_t M, const int32_t* slots, const float* weights, int32_t* state, int32_t* matched_len,
+                   int32_t min_match, int32_t* next_drafts, int32_t* next_n_draft, int32_t* chosen,
+                   void* workspace, int64_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------- diagnostics */
 

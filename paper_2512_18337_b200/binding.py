@@ -45,6 +45,9 @@ _SIGNATURES = {
     "sam_set_create": (C.c_int, [_vp, _i32, _vp, _i64, _vp, C.POINTER(_vp)]),
     "sam_set_refresh": (C.c_int, [_vp, _vp]),
     "sam_set_free": (None, [_vp]),
+    "sam_multi_workspace_bytes": (_i64, [_i32, _i32, _i32]),
+    "sam_multi_step": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp,
+                                 _i32, _vp, _vp, _vp, _vp, _i64, _vp]),
     "sam_multi_draft": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp]),
     "sam_argmax_partial": (C.c_int, [_vp, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sam_step_from_keys": (C.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]),
@@ -336,6 +339,22 @@ def sam_multi_draft(set_handle, B, M, slots, weights, state, matched_len, new_to
     _check(_load().sam_multi_draft(set_handle, B, M, _dev(slots), _dev(weights), _dev(state), _dev(matched_len),
                                    _dev(new_tokens), ld, _dev(n_new), K, min_match, _dev(drafts), _dev(n_draft),
                                    _dev(chosen), _stream(stream)), "sam_multi_draft")
+
+
+def sam_multi_workspace_bytes(B: int, K: int, M: int) -> int:
+    n = _load().sam_multi_workspace_bytes(B, K, M)
+    if n < 0:
+        raise SamError(int(n), "sam_multi_workspace_bytes")
+    return int(n)
+
+
+def sam_multi_step(set_handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,
+                   M, slots, weights, state, matched_len, min_match, next_drafts, next_n_draft, chosen,
+                   workspace, workspace_bytes, stream=None):
+    _check(_load().sam_multi_step(set_handle, _dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft),
+                                  _dev(argmax_out), _dev(accepted), _dev(n_accepted), M, _dev(slots), _dev(weights),
+                                  _dev(state), _dev(matched_len), min_match, _dev(next_drafts), _dev(next_n_draft),
+                                  _dev(chosen), _dev(workspace), workspace_bytes, _stream(stream)), "sam_multi_step")
 
 
 def sam_adaptive_switch(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:

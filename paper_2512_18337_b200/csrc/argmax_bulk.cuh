@@ -323,8 +323,19 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         // ------------------------------------------------------------------ walk-ahead warps
         if (pw.enabled) {
             const int w = warp - kBulkConsumerWarps - 2;
-            for (int b = blockIdx.x * kBulkWalkerWarps + w; b < pw.B; b += gridDim.x * kBulkWalkerWarps) {
-                prewalk_stream(sam, pw, b, lane);
+            const int per_stream = pw.M > 0 ? pw.M : 1;
+            for (int at = blockIdx.x * kBulkWalkerWarps + w; at < pw.B * per_stream; at += gridDim.x * kBulkWalkerWarps) {
+                const int b = at / per_stream;
+                if (pw.M > 0) {
+                    // composite drafting: this slot's own automaton (an empty slot has nothing to walk)
+                    const int member = __ldg(pw.slots + at);
+                    if (member >= 0 && member < pw.n_members) {
+                        const DeviceSam own = pw.table[member];
+                        prewalk_stream(own, pw, b, at, lane);
+                    }
+                    continue;
+                }
+                prewalk_stream(sam, pw, b, at, lane);
                 if (ft.mode != 0) {
                     // the walk-ahead is one of the stream's contributions; if it happens to be the last, finish here
                     int last = 0;

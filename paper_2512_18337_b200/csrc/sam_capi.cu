@@ -99,7 +99,7 @@ struct Scratch {
     int* n_rows;
     int64_t bytes;
 };
-Scratch scratch_layout(void* base, int32_t B, int32_t K) {
+Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M: automaton slots per stream (walk-ahead arrays)
     auto up = [](int64_t x) { return (x + 255) & ~int64_t(255); };
     const int64_t R = static_cast<int64_t>(B) * (K + 1);
     char* p = static_cast<char*>(base);
@@ -107,8 +107,8 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K) {
     int64_t o = 0;
     s.keys = reinterpret_cast<unsigned long long*>(p + o);  o = up(o + R * 8);
     s.status = reinterpret_cast<int*>(p + o);               o += 256;
-    s.pre_state = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * K * 4);
-    s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * K * 4);
+    s.pre_state = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * M * K * 4);
+    s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * M * K * 4);
     s.done = reinterpret_cast<int*>(p + o);                 o = up(o + static_cast<int64_t>(B) * 4);
     s.row_list = reinterpret_cast<int*>(p + o);             o = up(o + R * 4);
     s.n_rows = reinterpret_cast<int*>(p + o);               o += 256;
@@ -659,6 +659,69 @@ int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slo
         state, matched_len, new_tokens, ld, n_new, K, min_match, drafts, n_draft, chosen);
     SAM_CUDA(cudaGetLastError());
     ++g_launches;
+    return SAM_OK;
+}
+
+int64_t sam_multi_workspace_bytes(int32_t B, int32_t K, int32_t M) {
+    if (B < 0 || K < 1 || K > SAM_K_MAX || M < 1 || M > kMaxSlots) return SAM_ERR_INVALID_ARG;
+    return scratch_layout(nullptr, B, K, M).bytes;
+}
+
+int sam_multi_step(const sam_set* set,
+                   const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
+                   const int32_t* drafts, const int32_t* n_draft,
+                   int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
+                   int32_t M, const int32_t* slots, const float* weights, int32_t* state, int32_t* matched_len,
+                   int32_t min_match, int32_t* next_drafts, int32_t* next_n_draft, int32_t* chosen,
+                   void* workspace, int64_t workspace_bytes, void* cuda_stream) {
+    if (!set || M < 1 || M > kMaxSlots || min_match < 1) return SAM_ERR_INVALID_ARG;
+    if (B < 0 || K < 1 || K > SAM_K_MAX || V < 1 || row_stride_elems < V) return SAM_ERR_INVALID_ARG;
+    if (B == 0) return SAM_OK;
+    if (!logits_bf16 || !drafts || !n_draft || !argmax_out || !accepted || !n_accepted || !slots || !weights || !state ||
+        !matched_len || !next_drafts || !next_n_draft || !chosen || !workspace || !aligned(logits_bf16, 2) ||
+        !aligned(workspace, 8))
+        return SAM_ERR_INVALID_ARG;
+    if (workspace_bytes < sam_multi_workspace_bytes(B, K, M)) return SAM_ERR_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t R = static_cast<int64_t>(B) * (K + 1);
+    const Scratch sc = scratch_layout(workspace, B, K, M);
+    const DeviceSam* table = static_cast<const DeviceSam*>(set->device_buf);
+    const int n_members = static_cast<int>(set->members.size());
+    PreWalk pw{state, matched_len, drafts, n_draft, sc.pre_state, sc.pre_len, B, K, 1, 0, table, slots, M, n_members};
+    bool did_prewalk = false;
+    int rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, nullptr, &pw, &did_prewalk);
+    if (rc != SAM_OK) return rc;
+    if (!did_prewalk) {
+        // the direct-load argmax kernel has no spare warps: the slots walk the whole accepted run afterwards
+        const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                            argmax_out, accepted, n_accepted, sc.keys, nullptr, nullptr, 1, nullptr, nullptr,
+                            nullptr, nullptr, 0u, nullptr};
+        rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
+        if (rc != SAM_OK) return rc;
+        multi_draft_kernel<<<static_cast<unsigned>(B), 32 * M, 0, st>>>(
+            table, n_members, B, M, slots, weights, state, matched_len, accepted, K + 1, n_accepted, K, min_match,
+            next_drafts, next_n_draft, chosen);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+    } else {
+        const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
+                            argmax_out, accepted, n_accepted, sc.keys, nullptr, nullptr, min_match, next_drafts,
+                            next_n_draft, nullptr, nullptr, 0u, nullptr};
+        const MultiArgs ma{table, n_members, M, slots, weights, state, matched_len, sc.pre_state, sc.pre_len, chosen};
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(B));
+        cfg.blockDim = dim3(32 * M);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        SAM_CUDA(cudaLaunchKernelEx(&cfg, multi_step_kernel, aa, ma));
+        ++g_launches;
+    }
+    prof_mark(2, st);
+    prof_done();
     return SAM_OK;
 }
 

@@ -231,6 +231,23 @@ multi_draft_kernel(const DeviceSam* __restrict__ table, int n_members, int B, in
     }
 }
 
+// Composite step after the argmax: warp 0 accepts (decode, longest matching prefix, the model's own token),
+// then every slot resumes from the state its walk-ahead reached after the accepted prefix, follows the model's
+// token in its own automaton, and the slots compete for the next draft as in multi_draft_kernel.
+// Declared here, defined after accept_stream.
+struct AcceptArgs;
+struct MultiArgs {
+    const DeviceSam* table;
+    int n_members, M;
+    const int* slots;          // [B, M]
+    const float* weights;      // [B, M]
+    int* state;                // [B, M]
+    int* matched_len;          // [B, M]
+    const int* pre_state;      // [B, M, K]
+    const int* pre_len;        // [B, M, K]
+    int* chosen;               // [B]
+};
+
 // Walk-ahead along the draft.  While the logits of a step are still being reduced, spare warps
 // follow the automaton over each stream's DRAFT tokens and record the (state, matched_len)
 // reached after every prefix.  Whatever prefix the verification later accepts, the walk over it
@@ -245,11 +262,17 @@ struct PreWalk {
     int B, K;
     int enabled;
     int no_spec;             // speculation is off for this step: every proposal counts as empty
+    // composite drafting: M > 0 slots per stream, each with its own automaton and state;
+    // state / matched_len / pre_state / pre_len are then indexed by b * M + m
+    const DeviceSam* table;
+    const int* slots;        // [B, M] member number or -1
+    int M, n_members;
 };
 
-__device__ __forceinline__ void prewalk_stream(const DeviceSam& sam, const PreWalk& pw, int b, int lane) {
-    int s = pw.state[b];
-    int L = pw.matched_len[b];
+// `at` indexes the state arrays (b for a single automaton, b * M + m for a slot); the drafts are stream b's.
+__device__ __forceinline__ void prewalk_stream(const DeviceSam& sam, const PreWalk& pw, int b, int at, int lane) {
+    int s = pw.state[at];
+    int L = pw.matched_len[at];
     sanitize_stream_state(sam, s, L);
     const int nd = pw.no_spec ? 0 : max(0, min(pw.n_draft[b], pw.K));
     const int d = (lane < nd) ? pw.drafts[static_cast<long long>(b) * pw.K + lane] : -1;
@@ -262,8 +285,8 @@ __device__ __forceinline__ void prewalk_stream(const DeviceSam& sam, const PreWa
         if (lane == j) { my_s = s; my_L = L; }
     }
     if (lane < nd) {
-        pw.pre_state[static_cast<long long>(b) * pw.K + lane] = my_s;
-        pw.pre_len[static_cast<long long>(b) * pw.K + lane] = my_L;
+        pw.pre_state[static_cast<long long>(at) * pw.K + lane] = my_s;
+        pw.pre_len[static_cast<long long>(at) * pw.K + lane] = my_L;
     }
 }
 
@@ -526,7 +549,8 @@ struct AcceptArgs {
 // kAfterGrid: the kernel was launched as a programmatic dependent of the argmax kernel - everything that
 // does not depend on that kernel's output is loaded first, then the warp waits for it to finish.
 template <int kMode, bool kAfterGrid = false>
-__device__ __forceinline__ void accept_stream(const DeviceSam& sam, const AcceptArgs& p, int b, int lane) {
+__device__ __forceinline__ void accept_stream(const DeviceSam& sam, const AcceptArgs& p, int b, int lane,
+                                              int* out_a = nullptr, int* out_bonus = nullptr) {
     const int K = p.K;
     const int K1 = K + 1;
     const long long row0 = static_cast<long long>(b) * K1;
@@ -571,6 +595,8 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
     const int bonus_lo = __shfl_sync(kFull, am[0], a & 31);
     const int bonus_hi = __shfl_sync(kFull, am[1], 0);
     const int bonus = (a < 32) ? bonus_lo : bonus_hi;
+    if (out_a) *out_a = a;
+    if (out_bonus) *out_bonus = bonus;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int j = lane + 32 * h;
@@ -629,6 +655,72 @@ accept_kernel(DeviceSam sam, AcceptArgs p) {
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= p.B) return;
     accept_stream<kMode, true>(sam, p, b, lane);
+}
+
+__global__ void __launch_bounds__(32 * kMaxSlots)
+multi_step_kernel(AcceptArgs p, MultiArgs q) {
+    __shared__ float score[kMaxSlots];
+    __shared__ int ok[kMaxSlots];
+    __shared__ int winner, sh_a, sh_bonus;
+    const int b = blockIdx.x;
+    const int m = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int K = p.K;
+    const long long at = static_cast<long long>(b) * q.M + m;
+    // what does not depend on the argmax kernel
+    const int member = q.slots[at];
+    const bool live = member >= 0 && member < q.n_members;
+    int s = 0, L = 0;
+    RecRegs r = root_rec();
+    DeviceSam sam;
+    if (live) {
+        sam = q.table[member];
+        s = q.state[at];
+        L = q.matched_len[at];
+        sanitize_stream_state(sam, s, L);
+        if (s != 0) r = load_rec(sam, s);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (m == 0) {
+        int a = 0, bonus = 0;
+        accept_stream<kTailVerifyOnly>(DeviceSam{}, p, b, lane, &a, &bonus);
+        if (lane == 0) { sh_a = a; sh_bonus = bonus; }
+    }
+    __syncthreads();
+    const int a = sh_a, bonus = sh_bonus;
+    if (live) {
+        if (a > 0) {                                   // resume after the accepted prefix
+            s = __ldcg(q.pre_state + at * K + (a - 1));
+            L = __ldcg(q.pre_len + at * K + (a - 1));
+            r = (s > 0 && s < sam.n_states) ? load_rec(sam, s) : root_rec();
+            if (!(s > 0 && s < sam.n_states)) { s = 0; L = 0; }
+        }
+        walk_token(sam, bonus, s, L, r, lane);
+        if (lane == 0) {
+            q.state[at] = s;
+            q.matched_len[at] = L;
+        }
+    }
+    if (lane == 0) {
+        ok[m] = live && L >= p.min_match;
+        score[m] = live ? q.weights[at] * static_cast<float>(L) : 0.0f;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int w = -1;
+        float best = 0.0f;
+        for (int x = 0; x < q.M; ++x)
+            if (ok[x] && (w < 0 || score[x] > best)) { w = x; best = score[x]; }
+        winner = w;
+        q.chosen[b] = w;
+        if (w < 0) p.next_n_draft[b] = 0;
+    }
+    __syncthreads();
+    if (winner == m) {
+        const int nd = emit_draft(sam, L, r, K, p.min_match, p.next_drafts + static_cast<long long>(b) * K, lane);
+        if (lane == 0) p.next_n_draft[b] = nd;
+    } else if (winner < 0 && m == 0 && lane < K) {
+        p.next_drafts[static_cast<long long>(b) * K + lane] = -1;
+    }
 }
 
 }  // namespace samb200

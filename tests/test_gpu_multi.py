@@ -120,3 +120,62 @@ def test_multi_draft_argument_checks():
     args = (z.data_ptr(), f.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr(), 1, z.data_ptr())
     assert lib.sam_multi_draft(sset.handle, 1, 9, *args, 2, 1, z.data_ptr(), z.data_ptr(), z.data_ptr(), None) == -1   # M > 8
     assert lib.sam_multi_draft(sset.handle, 0, 1, *args, 2, 1, z.data_ptr(), z.data_ptr(), z.data_ptr(), None) == 0    # B = 0
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+def test_multi_step_closed_loop(variant):
+    """The fused composite step (argmax with every slot's walk-ahead riding along, accept, per-slot resume,
+    slot choice, next draft) against the oracle's accept followed by its composite drafting.  Variant 1 takes
+    the direct-load argmax kernel, which has no walk-ahead: the slots then walk the whole accepted run."""
+    rng = np.random.default_rng(11)
+    sep, B, M, K, mm, V = 999, 70, 3, 7, 2, 4096
+    corpora = [_corpus(rng, n, sep) for n in (5000, 3000, 4000, 2000)]
+    members_o = [oracle.OracleSAM(c, [sep]) for c in corpora]
+    sset = S.SamSet([S.SamIndex(c, [sep]) for c in corpora])
+    slots = rng.integers(-1, 4, size=(B, M)).astype(np.int32)
+    slots[0] = -1
+    weights = rng.choice(np.array([0.5, 1.0, 1.0, 2.0], np.float32), size=(B, M)).astype(np.float32)
+    st_o = np.zeros((B, M), np.int32); ml_o = np.zeros((B, M), np.int32)
+    i32 = dict(dtype=torch.int32, device=DEV)
+    st, ml = torch.zeros((B, M), **i32), torch.zeros((B, M), **i32)
+    d, nd, ch = torch.full((B, K), -9, **i32), torch.full((B,), -9, **i32), torch.full((B,), -9, **i32)
+    am, acc, nacc = torch.zeros((B, K + 1), **i32), torch.zeros((B, K + 1), **i32), torch.zeros(B, **i32)
+    sl_d, w_d = _dev(slots, np.int32), _dev(weights, np.float32)
+    wsb = S.sam_multi_workspace_bytes(B, K, M)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
+    S.sam_workspace_init(ws, wsb)
+    # prime every stream with a span of some member
+    toks = np.stack([members_o[int(rng.integers(0, 4))].corpus[s0:s0 + 10] for s0 in rng.integers(0, 1900, size=B)]).astype(np.int32)
+    n_new = np.full(B, 10, np.int32)
+    S.sam_multi_draft(sset.handle, B, M, sl_d, w_d, st, ml, _dev(toks, np.int32), 10, _dev(n_new, np.int32), K, mm, d, nd, ch)
+    d_o, nd_o, ch_o = oracle.multi_draft(members_o, slots, weights, st_o, ml_o, toks, n_new, K, mm)
+    torch.cuda.synchronize()
+    assert (d.cpu().numpy() == d_o).all() and (nd.cpu().numpy() == nd_o).all()
+    S.sam_set_argmax_variant(variant)
+    try:
+        full_accepts = 0
+        for step in range(10):
+            bits = W.f32_to_bf16_bits(rng.standard_normal((B * (K + 1), V), dtype=np.float32))
+            for b in range(B):
+                for j in range(int(nd_o[b]) + 1):
+                    # the "model" mostly continues the winning member's text, sometimes goes its own way
+                    if j < nd_o[b] and rng.random() < 0.8:
+                        bits[b * (K + 1) + j, d_o[b, j]] = 0x4200
+                    elif rng.random() < 0.5:
+                        c = members_o[int(rng.integers(0, 4))].corpus
+                        bits[b * (K + 1) + j, int(c[int(rng.integers(0, c.shape[0]))])] = 0x4200
+            lg = torch.from_numpy(bits.view(np.int16)).to(DEV).view(torch.bfloat16)
+            S.sam_multi_step(sset.handle, lg, V, B, K, V, d, nd, am, acc, nacc, M, sl_d, w_d, st, ml, mm, d, nd, ch, ws, wsb)
+            torch.cuda.synchronize()
+            am_o = oracle.argmax_batch(bits).reshape(B, K + 1)
+            acc_o, nacc_o = oracle.accept_batch(d_o, nd_o, am_o)
+            full_accepts += int(((nacc_o - 1 == nd_o) & (nd_o > 0)).sum())
+            d_o, nd_o, ch_o = oracle.multi_draft(members_o, slots, weights, st_o, ml_o, acc_o, nacc_o, K, mm)
+            assert (am.cpu().numpy() == am_o).all(), step
+            assert (acc.cpu().numpy() == acc_o).all() and (nacc.cpu().numpy() == nacc_o).all(), step
+            assert (st.cpu().numpy() == st_o).all() and (ml.cpu().numpy() == ml_o).all(), step
+            assert (ch.cpu().numpy() == ch_o).all(), step
+            assert (nd.cpu().numpy() == nd_o).all() and (d.cpu().numpy() == d_o).all(), step
+        assert full_accepts > 0
+    finally:
+        S.sam_set_argmax_variant(0)
