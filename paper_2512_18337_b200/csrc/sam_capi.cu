@@ -186,9 +186,16 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
 }
 
 template <int kMode>
-int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st) {
+int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st, bool after_own_argmax = true) {
     const int warps = 4;
     const unsigned grid = static_cast<unsigned>((a.B + warps - 1) / warps);
+    if (!after_own_argmax) {
+        // whatever precedes in the stream may still be producing this kernel's inputs: ordinary stream order
+        accept_kernel<kMode><<<grid, warps * 32, 0, st>>>(sam, a);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+        return SAM_OK;
+    }
     // launched as a programmatic dependent of the kernel before it in the stream (the argmax kernel): its
     // blocks are placed, and load what does not depend on that kernel, while that kernel is still running
     cudaLaunchConfig_t cfg = {};
@@ -604,7 +611,7 @@ int sam_step_from_keys(const sam_index* idx, int64_t* keys, int32_t B, int32_t K
     const AcceptArgs aa{nullptr, 0, B, K, drafts, n_draft, argmax_out, accepted, n_accepted,
                         reinterpret_cast<unsigned long long*>(keys), state, matched_len, min_match, next_drafts,
                         next_n_draft, nullptr, nullptr, 0u, nullptr};
-    return launch_accept<kTailFullWalk>(idx->dev, aa, static_cast<cudaStream_t>(cuda_stream));
+    return launch_accept<kTailFullWalk>(idx->dev, aa, static_cast<cudaStream_t>(cuda_stream), false);
 }
 
 int64_t sam_set_bytes(int32_t n_members) {
