@@ -152,6 +152,8 @@ def run_ours(args):
     S.sam_set_argmax_variant(args.variant)
 
     base = W.CONFIGS[args.config]
+    if args.streams > 0:
+        base = base.scaled(B=args.streams, name=f"{base.name}_B{args.streams}")
     # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
     # read-only automaton is replicated; no data-path collective
     cfg = base.scaled(steps=args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1)
@@ -726,7 +728,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (default: B=256, K=16)")
+    ap.add_argument("--config", type=int, default=2, help="workload index 0..5 (default 2: B=256, K=16; 5: the paper's evaluation shape, B=4, K=3)")
+    ap.add_argument("--streams", type=int, default=0, help="override the workload's number of streams B (per GPU)")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--presleep-cycles", type=int, default=300000,
                     help="length of the spin kernel enqueued before each timed step (outside the events)")

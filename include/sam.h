@@ -391,9 +391,9 @@ int sam_multi_step(const sam_set* set,
  * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
 int sam_profile_enable(int32_t max_calls);
 /* Selects the kernels of sam_verify / sam_step for later calls (process-wide; for measurements
- * and tests): 0 = by alignment (default: a bulk-copy pipelined argmax kernel when the logits base
- * and row stride are 16-byte aligned, a direct-load kernel otherwise, each followed by the accept
- * kernel), 1 = always direct loads, 2 = as 0, but the bulk-copy kernel also runs the accept step of
+ * and tests): 0 = automatic (default: a bulk-copy pipelined argmax kernel when the logits base
+ * and row stride are 16-byte aligned, a direct-load kernel otherwise or when K <= 4 and the logits
+ * are under 96 MiB, each followed by the accept kernel), 1 = always direct loads, 2 = as 0, but the bulk-copy kernel also runs the accept step of
  * every stream as soon as its rows are complete (one launch per call; measured slightly slower than
  * two launches on B200), 3 = same as 0. */
 int sam_set_argmax_variant(int32_t variant);

@@ -124,12 +124,17 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
                   int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
                   bool* did_prewalk = nullptr, const AcceptArgs* tail = nullptr, int tail_mode = 0,
                   int* done = nullptr, bool* did_tail = nullptr, const RowMap* rmap = nullptr) {
+    // Short proposals over little data (the paper's own setting: batch 4, three speculative tokens) are a latency
+    // case: the direct-load kernel starts faster than the bulk-copy pipeline and there is little for a walk-ahead to
+    // save (measured at K = 3: 12.2 vs 13.4 us per step for 4 streams, 25.2 vs 26.5 us for 64; equal near 200 MB of logits).
+    const bool latency_case = g_argmax_variant == 0 && tail != nullptr && tail->K <= 4 &&
+                              R * static_cast<int64_t>(V) * 2 <= (int64_t(96) << 20);
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != SAM_OK) return rc;
     const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0;
-    const bool bulk = rows_aligned && g_argmax_variant != 1;
+    const bool bulk = rows_aligned && g_argmax_variant != 1 && !latency_case;
     const RowMap rm = rmap ? *rmap : RowMap{nullptr, nullptr, 0};
     if (did_prewalk) *did_prewalk = false;
     if (did_tail) *did_tail = false;

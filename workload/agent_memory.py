@@ -78,6 +78,10 @@ CONFIGS: List[WorkloadConfig] = [
                    B=512, steps=8, K=16, min_match=2, accept_p=0.5, tie_frac=0.01, seed=3),
     WorkloadConfig("cfg4_long_trace", 8192, 8192, 151936, 1.05, 0.70, 32, 1024,
                    B=1024, steps=64, K=32, min_match=4, accept_p=0.7, tie_frac=0.0, seed=4),
+    # the shape of the paper's own evaluation (Section 6.5: batch size 4, one autoregressive + three speculative
+    # tokens per step), on the 1M-token corpus: a latency case, not a bandwidth case
+    WorkloadConfig("cfg5_paper_eval_shape_B4_K3", 256, 4096, 151936, 1.1, 0.40, 16, 256,
+                   B=4, steps=64, K=3, min_match=2, accept_p=0.7, tie_frac=0.0, seed=5),
 ]
 
 
