@@ -156,7 +156,10 @@ def run_ours(args):
         base = base.scaled(B=args.streams, name=f"{base.name}_B{args.streams}")
     # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
     # read-only automaton is replicated; no data-path collective
-    cfg = base.scaled(steps=args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1)
+    n_script_steps = args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1
+    if args.cpu_baseline and world == 1:
+        n_script_steps = max(n_script_steps, args.cpu_steps + 8)      # the oracle leg replays the same scripts from step 0
+    cfg = base.scaled(steps=n_script_steps)
     stream_cfg = cfg.scaled(seed=cfg.seed + 7919 * rank) if rank > 0 else cfg
 
     t0 = time.time()
@@ -380,7 +383,8 @@ def run_ours(args):
                                     "note": "the same bytes over the event bracket of the whole step in the timed region "
                                             "(argmax + accept + walk + draft)"}},
         "walk": walk,
-        "ote": st["ote"], "shr": st["shr"], "mean_n_draft": st["mean_n_draft"],
+        "ote": st["ote"], "shr": st["shr"], "shr_per_K_of_nonempty_proposals": st["shr_k"],
+        "mean_n_draft": st["mean_n_draft"],
         "device_counters": {"passes": dev_counters[0], "committed": dev_counters[1], "proposed": dev_counters[2],
                             "accepted_drafts": dev_counters[3], "nonempty_proposals": dev_counters[4],
                             "rows_read": dev_counters[5], "ote": dev_counters[1] / max(1, dev_counters[0]),
@@ -400,8 +404,9 @@ def run_ours(args):
 
 
 # ----------------------------------------------------------------------------- oracle arm
-def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads):
-    """Times the oracle's step (wall clock, planting excluded) on the same closed loop."""
+def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads, single_thread_steps=0):
+    """Times the oracle's step (wall clock, planting excluded) on the same closed loop; optionally goes on for a
+    few steps on one thread.  Returns (tokens, seconds, build seconds[, single-thread tokens, seconds])."""
     import oracle
     from tests.oracle_backend import OracleBackend
     feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
@@ -410,8 +415,10 @@ def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads)
     t_build = time.time() - t0
     toks, n = feeder.prime_tokens()
     drafts, n_draft = be.prime(toks, n)
-    tokens, secs = 0, 0.0
-    for t in range(warmup + steps):
+    tokens, secs, tokens1, secs1 = 0, 0.0, 0, 0.0
+    for t in range(warmup + steps + single_thread_steps):
+        if t == warmup + steps:
+            be.threads = 1
         ow = feeder.overwrites(t, drafts, n_draft)
         keep = np.arange(ow["row"].shape[0])
         saved = be.poke(ow["row"], ow["col"], ow["bits"], keep)
@@ -421,9 +428,14 @@ def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads)
         be.unpoke(ow["row"], ow["col"], saved)
         feeder.advance(out["n_accepted"])
         drafts, n_draft = out["drafts"], out["n_draft"]
-        if t >= warmup:
+        if t >= warmup + steps:
+            tokens1 += int(out["n_accepted"].sum())
+            secs1 += c1 - c0
+        elif t >= warmup:
             tokens += int(out["n_accepted"].sum())
             secs += c1 - c0
+    if single_thread_steps > 0:
+        return tokens, secs, t_build, tokens1, secs1
     return tokens, secs, t_build
 
 
@@ -431,8 +443,10 @@ def cpu_baseline(cfg, corpus, scripts, logits_dev, rowmax, steps):
     import oracle
     host_bits = W.device_bits_to_host(logits_dev)
     threads = oracle.host_threads()
-    tokens, secs, t_build = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, 1, steps, threads)
+    tokens, secs, t_build, tokens1, secs1 = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, 1, steps, threads, 4)
     return {"value": tokens / secs, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "single_thread": {"value": tokens1 / secs1, "unit": UNIT, "steps": 4,
+                              "argmax_GBps": cfg.rows * cfg.vocab * 2 * 4 / secs1 / 1e9},
             "sample": f"all {cfg.B} streams, first {steps} closed-loop steps after 1 warm-up step "
                       f"({secs:.2f} s of oracle stepping; oracle automaton build {t_build:.1f} s not included)",
             "ms_per_step": secs / steps * 1e3,
