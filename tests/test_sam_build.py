@@ -184,3 +184,31 @@ def test_argument_checks_that_need_no_device():
     finally:
         S.sam_free(h)
     assert S.sam_strerror(-3).startswith("automaton not uploaded")
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    """There is no CPU fallback: with the shared library absent the first call raises, and nothing under
+    the package imports the oracle."""
+    import subprocess
+    import sys
+    code = (
+        "import os, sys\n"
+        f"sys.path.insert(0, {ROOT!r})\n"
+        f"os.environ['SAM_B200_LIB'] = {str(tmp_path / 'nowhere.so')!r}\n"
+        "import numpy as np\n"
+        "import paper_2512_18337_b200 as S\n"
+        "try:\n"
+        "    S.sam_build(np.array([1, 2, 3], np.int32), [9])\n"
+        "except RuntimeError as e:\n"
+        "    assert 'missing' in str(e) and 'no CPU fallback' in str(e), e\n"
+        "    assert 'oracle' not in sys.modules\n"
+        "    print('raised')\n"
+    )
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0 and "raised" in out.stdout, out.stderr
+    # the product sources never import the oracle package
+    pkg = os.path.join(ROOT, "paper_2512_18337_b200")
+    for name in os.listdir(pkg):
+        if name.endswith(".py"):
+            text = open(os.path.join(pkg, name)).read()
+            assert "import oracle" not in text and "from oracle" not in text, name
