@@ -503,7 +503,7 @@ def run_growing(args):
     cfg = base.scaled(steps=args.warmup + args.steps + 1)
     corpus, logits, rowmax = make_inputs_gpu(cfg, device)
     scripts = W.make_scripts(cfg, corpus)
-    room = (cfg.K + 2) * cfg.B * (args.warmup + args.steps + 2) + (1 << 20)
+    room = (cfg.K + 2) * cfg.B * (args.warmup + args.steps + 2) + (1 << 20) + 32768
     t0 = time.time()
     index = S.SamIndex(corpus, [cfg.separator], device=device, max_tokens=cfg.n_corpus + room, max_token_id=cfg.separator)
     t_build_upload = time.time() - t0
@@ -516,6 +516,15 @@ def run_growing(args):
     S.sam_sync(index.handle)
     torch.cuda.synchronize()
     t_first_sync = time.time() - t0
+    # a 30k-token prompt arriving at once (the paper's asynchronous-construction experiment uses such a prompt):
+    # time until the builder thread has indexed it and the device copy is up to date
+    prompt = W.make_corpus(cfg.scaled(sessions=8, seed=cfg.seed + 202))[:30000]
+    t0 = time.time()
+    S.sam_extend(index.handle, prompt)
+    t_prompt_build = time.time() - t0
+    S.sam_sync(index.handle)
+    torch.cuda.synchronize()
+    t_prompt_total = time.time() - t0
     stats0 = S.sam_update_stats(index.handle)
 
     feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
@@ -566,6 +575,8 @@ def run_growing(args):
         "updates": {"incremental": stats1[0] - stats0[0], "full_images": stats1[1] - stats0[1],
                     "h2d_bytes_per_step": (stats1[2] - stats0[2]) / args.steps},
         "builder_thread_tokens_per_s": extra.shape[0] / t_extend,
+        "prompt_30k_tokens": {"indexed_on_host_ms": t_prompt_build * 1e3, "visible_on_device_ms": t_prompt_total * 1e3,
+                              "note": "drafting from the older text goes on meanwhile; nothing on the decoding path waits"},
         "first_sync_s": t_first_sync, "first_sync_bytes": stats0[2], "build_and_upload_s": t_build_upload,
         "device_bytes": index.device_bytes,
     }))
