@@ -100,11 +100,19 @@ bool pack_state(DynIndex& D, int32_t s, StateRec* r, const std::pair<int32_t, in
     r->e[0] = r->e[1] = r->e[2] = r->e[3] = -1;
     const int32_t d = b.deg[s];
     if (d <= 2) {
+        // the common case by far: read the one or two chain nodes directly
         if (d >= 1) {
-            b.sorted_row(s, tmp);
-            r->e[0] = tmp[0].first;
-            r->e[1] = tmp[0].second;
-            if (d == 2) { r->e[2] = tmp[1].first; r->e[3] = tmp[1].second; }
+            const int32_t x0 = b.head[s];
+            if (d == 1) {
+                r->e[0] = b.e_tok[x0];
+                r->e[1] = b.e_dst[x0];
+            } else {
+                const int32_t x1 = b.e_next[x0];
+                const bool swap = b.e_tok[x1] < b.e_tok[x0];
+                const int32_t lo = swap ? x1 : x0, hi = swap ? x0 : x1;
+                r->e[0] = b.e_tok[lo]; r->e[1] = b.e_dst[lo];
+                r->e[2] = b.e_tok[hi]; r->e[3] = b.e_dst[hi];
+            }
         }
         return true;
     }
@@ -232,10 +240,14 @@ int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
         *out = std::move(fresh);
         return rc;
     }
+    std::sort(b.dirty.begin(), b.dirty.end());      // new states are consecutive: mostly sequential memory from here on
     for (int32_t s : b.dirty) {
         StateRec r;
-        const auto lo = std::lower_bound(b.redirected.begin(), b.redirected.end(), std::make_pair(s, INT32_MIN));
-        const auto hi = std::lower_bound(lo, b.redirected.end(), std::make_pair(s + 1, INT32_MIN));
+        auto lo = b.redirected.end(), hi = b.redirected.end();
+        if (b.deg[s] >= 3) {                         // inline records are rebuilt from the chain; only rows need the list
+            lo = std::lower_bound(b.redirected.begin(), b.redirected.end(), std::make_pair(s, INT32_MIN));
+            hi = std::lower_bound(lo, b.redirected.end(), std::make_pair(s + 1, INT32_MIN));
+        }
         if (!pack_state(D, s, &r, lo == hi ? nullptr : &*lo, static_cast<size_t>(hi - lo), tmp, out)) {
             // wide area exhausted: lay everything out afresh and send the whole image instead
             Delta fresh;
