@@ -97,7 +97,7 @@ int64_t sam_workspace_bytes(int32_t B, int32_t K);
  * must not overlap on the device. */
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
 
-/* Reads the status word the verification kernels keep at the end of the scratch: 0 = fine,
+/* Reads the status word the verification kernels keep inside the scratch: 0 = fine,
  * 1 = a kernel gave up on one of its internal (bounded) waits, 2 = a kernel was handed more
  * finished streams than its internal queue holds (the host sizes the launch so that this does not
  * happen).  After a non-zero status the outputs of that call are not valid - re-initialise the
