@@ -65,7 +65,7 @@ def _check_verify(bits, V, B, K, rng):
     (1, 0, 3, 1), (7, 0, 3, 2), (8, 0, 2, 3), (9, 7, 5, 4), (1000, 0, 4, 8), (1000, 3, 4, 8),
     (4097, 0, 6, 5), (4097, 8, 6, 5), (50257, 0, 3, 7), (50257, 1, 3, 7), (151936, 0, 2, 8),
     (151936, 8, 3, 32), (8192 * 3, 0, 40, 16), (8191, 1, 33, 31), (8192 * 13 + 24, 0, 7, 3), (8192 * 12, 8, 9, 2),
-    (3, 5, 300, 1), (8200, 0, 1, 1), (8192 * 25 + 5, 3, 2, 2), (32768 * 3, 0, 5, 2), (32768 * 2 + 8, 0, 4, 1), (32768 * 2 - 3, 3, 4, 1),
+    (3, 5, 300, 1), (8200, 0, 1, 1), (1000003, 5, 2, 3), (1 << 20, 0, 1, 1), (8192 * 25 + 5, 3, 2, 2), (32768 * 3, 0, 5, 2), (32768 * 2 + 8, 0, 4, 1), (32768 * 2 - 3, 3, 4, 1),
 ])
 def test_verify_parity_shapes(V, pad, B, K):
     """Row lengths around vector/tile edges, misaligned row strides, every K edge."""
@@ -205,6 +205,32 @@ def test_draft_random_feeds(K, mm):
         assert (st == st_o).all() and (ml == ml_o).all()
         assert (nd == nd_o).all() and (d == d_o).all()
     assert (nd_o == 0).any() and (nd_o == K).any()
+
+
+@pytest.mark.parametrize("n_sep", [0, 1, 16])
+def test_draft_with_no_one_and_sixteen_separators(n_sep):
+    """The largest number of separator ids, a single one, and none at all (drafts then only end at the corpus end)."""
+    rng = np.random.default_rng(40 + n_sep)
+    corpus = rng.integers(0, 60, size=5000).astype(np.int32)
+    seps = list(range(100, 100 + n_sep))
+    if n_sep:
+        corpus[rng.integers(0, 5000, size=400)] = rng.choice(np.array(seps, np.int32), size=400)
+    index = S.SamIndex(corpus, seps)
+    osam = oracle.OracleSAM(corpus, seps if n_sep else np.zeros(0, np.int32))
+    B, ld, K, mm = 40, 8, 12, 1
+    st = np.zeros(B, np.int32); ml = np.zeros(B, np.int32)
+    st_o = st.copy(); ml_o = ml.copy()
+    cut_short = 0
+    for step in range(4):
+        starts = rng.integers(0, 5000 - ld, size=B)
+        starts[:4] = 5000 - ld                                   # runs into the corpus end
+        toks = np.stack([corpus[s0:s0 + ld] for s0 in starts]).astype(np.int32)
+        n_new = rng.integers(1, ld + 1, size=B).astype(np.int32)
+        d_o, nd_o = osam.draft_batch(st_o, ml_o, toks, n_new, K, mm)
+        st, ml, d, nd = _draft_gpu(index, B, st, ml, toks, n_new, K, mm)
+        assert (st == st_o).all() and (ml == ml_o).all() and (nd == nd_o).all() and (d == d_o).all()
+        cut_short += int(((nd_o < K) & (ml_o >= mm)).sum())
+    assert cut_short > 0
 
 
 def test_draft_rejects_foreign_state():
