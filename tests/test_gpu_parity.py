@@ -316,3 +316,48 @@ def test_closed_loop_scaled_configs(i, kw):
     cfg = W.CONFIGS[i].scaled(**kw)
     tr_o, tr_g = _closed_loop_pair(cfg)
     _assert_traces_equal(tr_o, tr_g)
+
+
+def _colliding_tokens(log2cap, count, limit=1 << 20):
+    """Token ids whose home slot in a hash row of 2^log2cap slots is the same (multiplicative hashing with the
+    golden-ratio constant - the row layout documented for states with more than 32 transitions)."""
+    tok = np.arange(1, limit, dtype=np.uint64)
+    home = ((tok * np.uint64(0x9E3779B1)) & np.uint64(0xFFFFFFFF)) >> np.uint64(32 - log2cap)
+    same = tok[home == home[0]][:count]
+    assert same.shape[0] == count
+    return same.astype(np.int32)
+
+
+@pytest.mark.parametrize("growing", [False, True])
+def test_hash_row_with_a_probe_run_longer_than_one_window(growing):
+    """A hub state whose 40 successors all hash to the same slot: the lookup has to go on into a second
+    32-slot window, both for successors that are there and for a token that is not."""
+    log2cap = 8 if growing else 7            # 40 transitions: 128 slots in a fixed index, 256 in a growing one
+    succ = _colliding_tokens(log2cap, 41)
+    present, absent = succ[:40], int(succ[40])
+    hub, sep = 5, 3
+    corpus = np.empty(2 * 40, np.int32)
+    corpus[0::2] = hub
+    corpus[1::2] = present
+    if growing:
+        index = S.SamIndex(corpus[:20], [sep], max_tokens=1000, max_token_id=int(succ.max()))
+        S.sam_extend(index.handle, corpus[20:])
+        S.sam_sync(index.handle)
+    else:
+        index = S.SamIndex(corpus, [sep])
+    osam = oracle.OracleSAM(corpus, [sep])
+    ex = osam.export()
+    s_hub, _ = osam.walk(0, 0, [hub])
+    assert ex["row_ptr"][s_hub + 1] - ex["row_ptr"][s_hub] == 40
+    B = 42
+    toks = np.full((B, 2), hub, np.int32)
+    toks[:40, 1] = present
+    toks[40, 1] = absent                     # same home slot, not a successor: falls back through the suffix link
+    toks[41, 1] = hub
+    n_new = np.full(B, 2, np.int32)
+    st = np.zeros(B, np.int32); ml = np.zeros(B, np.int32)
+    st_o = st.copy(); ml_o = ml.copy()
+    d_o, nd_o = osam.draft_batch(st_o, ml_o, toks, n_new, 4, 1)
+    st, ml, d, nd = _draft_gpu(index, B, st, ml, toks, n_new, 4, 1)
+    assert (st == st_o).all() and (ml == ml_o).all() and (nd == nd_o).all() and (d == d_o).all()
+    assert (ml_o[:40] == 2).all() and ml_o[40] == 0
