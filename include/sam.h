@@ -359,6 +359,11 @@ int sam_set_create(const sam_index* const* members, int32_t n_members, void* dev
                    void* cuda_stream, sam_set** out);
 int sam_set_refresh(sam_set* set, void* cuda_stream);
 void sam_set_free(sam_set* set);
+/* sam_renormalize for composite state: after member number `member` has grown (sam_sync, sam_set_refresh),
+ * every slot that names it is moved to the state that now holds its string; other slots are untouched.
+ * slots, state, matched_len: device [B, M]. */
+int sam_set_renormalize(const sam_set* set, int32_t member, int32_t B, int32_t M, const int32_t* slots,
+                        int32_t* state, const int32_t* matched_len, void* cuda_stream);
 int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slots, const float* weights,
                     int32_t* state, int32_t* matched_len, const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
                     int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, int32_t* chosen,

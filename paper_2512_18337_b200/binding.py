@@ -45,6 +45,7 @@ _SIGNATURES = {
     "sam_set_create": (C.c_int, [_vp, _i32, _vp, _i64, _vp, C.POINTER(_vp)]),
     "sam_set_refresh": (C.c_int, [_vp, _vp]),
     "sam_set_free": (None, [_vp]),
+    "sam_set_renormalize": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp]),
     "sam_multi_workspace_bytes": (_i64, [_i32, _i32, _i32]),
     "sam_multi_step": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp,
                                  _i32, _vp, _vp, _vp, _vp, _i64, _vp]),
@@ -321,6 +322,11 @@ class SamSet:
 
     def refresh(self, stream=None):
         _check(_load().sam_set_refresh(self.handle, _stream(stream)), "sam_set_refresh")
+
+    def renormalize(self, member: int, B: int, M: int, slots, state, matched_len, stream=None):
+        """After member `member` has grown and refresh() was called: repair the slots that name it."""
+        _check(_load().sam_set_renormalize(self.handle, member, B, M, _dev(slots), _dev(state), _dev(matched_len),
+                                           _stream(stream)), "sam_set_renormalize")
 
     def close(self):
         h, self.handle = self.handle, None

@@ -657,6 +657,22 @@ int sam_set_create(const sam_index* const* members, int32_t n_members, void* dev
 
 void sam_set_free(sam_set* set) { delete set; }
 
+int sam_set_renormalize(const sam_set* set, int32_t member, int32_t B, int32_t M, const int32_t* slots,
+                        int32_t* state, const int32_t* matched_len, void* cuda_stream) {
+    if (!set || member < 0 || member >= static_cast<int32_t>(set->members.size()) || B < 0 || M < 1 || M > kMaxSlots)
+        return SAM_ERR_INVALID_ARG;
+    const sam_index* idx = set->members[member];
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B == 0) return SAM_OK;
+    if (!slots || !state || !matched_len) return SAM_ERR_INVALID_ARG;
+    const int n = B * M;
+    renormalize_slots_kernel<<<static_cast<unsigned>((n + 127) / 128), 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        idx->dev, member, n, slots, state, matched_len);
+    SAM_CUDA(cudaGetLastError());
+    ++g_launches;
+    return SAM_OK;
+}
+
 int sam_multi_draft(const sam_set* set, int32_t B, int32_t M, const int32_t* slots, const float* weights,
                     int32_t* state, int32_t* matched_len, const int32_t* new_tokens, int32_t ld, const int32_t* n_new,
                     int32_t K, int32_t min_match, int32_t* drafts, int32_t* n_draft, int32_t* chosen,

@@ -74,4 +74,25 @@ renormalize_kernel(DeviceSam sam, int B, int* __restrict__ state, const int* __r
     if (s != s0) state[b] = s;
 }
 
+// The same for composite drafting: only the slots that name `member` are touched (slots, state and
+// matched_len are [n] = B * M entries).
+__global__ void __launch_bounds__(128)
+renormalize_slots_kernel(DeviceSam sam, int member, int n, const int* __restrict__ slots, int* __restrict__ state,
+                         const int* __restrict__ matched_len) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n || slots[i] != member) return;
+    int s = state[i];
+    const int L = matched_len[i];
+    if (s <= 0 || s >= sam.n_states || L < 0) return;
+    const int s0 = s;
+    for (int hop = 0; hop < (1 << 30) && s != 0; ++hop) {
+        const int link = __ldg(&sam.rec[s].link);
+        if (link < 0 || link >= sam.n_states) break;
+        const int link_len = (link == 0) ? 0 : __ldg(&sam.rec[link].len);
+        if (L > link_len) break;
+        s = link;
+    }
+    if (s != s0) state[i] = s;
+}
+
 }  // namespace samb200

@@ -100,12 +100,8 @@ def test_multi_draft_parity_with_growth_and_verification():
                 col_o = np.ascontiguousarray(st_o[own, m])
                 members_o[4].renormalize(col_o, np.ascontiguousarray(ml_o[own, m]))
                 st_o[own, m] = col_o
-            # on the device the member's states are gathered, renormalised and scattered back
-            own_d = (sl_d == 4).view(-1).nonzero().view(-1)
-            sub_s, sub_l = st.view(-1)[own_d].contiguous(), ml.view(-1)[own_d].contiguous()
-            S.sam_renormalize(members_g[4].handle, int(own_d.numel()), sub_s, sub_l)
+            sset.renormalize(4, B, M, sl_d, st, ml)
             torch.cuda.synchronize()
-            st.view(-1)[own_d] = sub_s
             assert (st.cpu().numpy() == st_o).all()
     assert seen_slots >= {-1, 0, 1, 2, 3}
 
