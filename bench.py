@@ -36,7 +36,7 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
 # capture summarised in profiles/launch_list_cfg2.md (config 2, argmax_bulk_kernel; traffic scales with rows)
-NCU_DRAM_BYTES_PER_ROW = 304335.1
+NCU_DRAM_BYTES_PER_ROW = 304325.1
 # dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
 NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 46.9
 
