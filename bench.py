@@ -218,6 +218,18 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
+    graph_launches = None
+    direct_launch = be.launch_step
+    if args.graph:
+        # the step's launches recorded once (after ordinary calls have done the first-use set-up) and replayed:
+        # same kernels, same buffers, no per-launch host work and no gaps between the two kernels
+        l0 = S.sam_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            direct_launch()
+        graph_launches = S.sam_launch_count() - l0
+        be.launch_step = graph.replay
+        torch.cuda.synchronize()
     launches0 = S.sam_launch_count()
     be.counters.zero_()
     torch.cuda.synchronize()
@@ -229,6 +241,9 @@ def run_ours(args):
         dist.barrier()
     wall = time.time() - wall0
     launches = S.sam_launch_count() - launches0
+    if args.graph:
+        launches = graph_launches * args.steps      # kernel nodes of the replayed graph
+        be.launch_step = direct_launch
     dev_counters = [int(x) for x in be.counters.cpu().numpy()]
     clocks = sampler.stop(wall0, wall0 + wall) if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
@@ -325,6 +340,29 @@ def run_ours(args):
                                            "cross the bus (a different contract: the other rows are not arg-maxed)"}}
         del staging, host_logits
 
+    # ---- with --graph: what a serving loop that issues steps back to back sees, direct calls against replays of
+    # the recorded step (one event pair around the whole run; the logits stay as they are, so most drafts are
+    # rejected, but every row is arg-maxed and every stream accepted, walked and drafted as in any other step)
+    back_to_back = None
+    if args.graph:
+        n_b2b = 300
+        back_to_back = {"steps": n_b2b}
+        for name, fn in (("direct_calls_us_per_step", direct_launch), ("graph_replay_us_per_step", graph.replay)):
+            for _ in range(10):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            w0 = time.perf_counter()
+            e0.record()
+            for _ in range(n_b2b):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            w1 = time.perf_counter()
+            back_to_back[name] = e0.elapsed_time(e1) * 1e3 / n_b2b
+            back_to_back[name.replace("_us_per_step", "_wall_us_per_step")] = (w1 - w0) * 1e6 / n_b2b
+        assert be.status() == 0
+
     all_tokens, max_ms = reduce_over_ranks(tokens, total_ms, world, device)
     if rank != 0:
         if world > 1:
@@ -373,7 +411,7 @@ def run_ours(args):
         "steps_per_s": args.steps / (max_ms / 1e3),
         "stream_steps_per_s": world * cfg.B * args.steps / (max_ms / 1e3),
         "gpu_launches": launches,
-        "launches_per_step": launches_per_step, "variant": args.variant,
+        "launches_per_step": launches_per_step, "variant": args.variant, "cuda_graph": bool(args.graph), "back_to_back": back_to_back,
         "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
                      "traffic": (NCU_DRAM_BYTES_PER_ROW * (rows_read_per_step if args.skip_unused_rows else R)) if NCU_DRAM_BYTES_PER_ROW else None,
@@ -774,6 +812,8 @@ def main():
     ap.add_argument("--multi", type=int, default=0,
                     help="> 0: closed loop with composite drafting over that many member automata (1..8); separate JSON line")
     ap.add_argument("--multi-unfused", action="store_true", help="with --multi: sam_verify + sam_multi_draft instead of sam_multi_step")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one sam_step in a CUDA graph after the warm-up and replay it for every timed step")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
     args = ap.parse_args()

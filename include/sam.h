@@ -23,6 +23,10 @@
  *     the caller; a new stream starts at (0, 0).
  *   - There is no CPU fallback: without a usable CUDA device the hot-path calls fail with
  *     SAM_ERR_CUDA.
+ *   - sam_step / sam_step_ex may be recorded in a CUDA graph by stream capture and replayed (tested:
+ *     the replayed step gives the oracle's trace).  Make one ordinary call on the device first (it
+ *     does the library's first-use set-up); the recorded launches keep the pointers, sizes and
+ *     options of the recorded call, and replays share its scratch, so they must not overlap.
  */
 #ifndef SAM_B200_H
 #define SAM_B200_H
