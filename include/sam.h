@@ -23,6 +23,10 @@
  *     the caller; a new stream starts at (0, 0).
  *   - There is no CPU fallback: without a usable CUDA device the hot-path calls fail with
  *     SAM_ERR_CUDA.
+ *   - Calls may come from several host threads at once, on different streams, as long as they share
+ *     neither scratch nor output buffers (one handle may serve them all: hot-path calls only read it).
+ *     The diagnostic switches (sam_profile_*, sam_set_argmax_variant) are process-wide and not for
+ *     concurrent use.
  *   - sam_step / sam_step_ex may be recorded in a CUDA graph by stream capture and replayed (tested:
  *     the replayed step gives the oracle's trace).  Make one ordinary call on the device first (it
  *     does the library's first-use set-up); the recorded launches keep the pointers, sizes and

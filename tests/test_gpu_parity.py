@@ -361,3 +361,44 @@ def test_hash_row_with_a_probe_run_longer_than_one_window(growing):
     st, ml, d, nd = _draft_gpu(index, B, st, ml, toks, n_new, 4, 1)
     assert (st == st_o).all() and (ml == ml_o).all() and (nd == nd_o).all() and (d == d_o).all()
     assert (ml_o[:40] == 2).all() and ml_o[40] == 0
+
+
+def test_two_host_threads_on_two_streams():
+    """Two host threads drive two independent closed loops at once, each on a stream and a scratch of its own, over
+    one shared automaton: calls from several threads are allowed as long as they do not share scratch or outputs."""
+    import threading
+    cfgs = [W.CONFIGS[2].scaled(sessions=64, B=40, steps=10), W.CONFIGS[2].scaled(sessions=64, B=24, steps=10, seed=77)]
+    corpus = W.make_corpus(cfgs[0])                      # one text; the second loop differs in streams, scripts and logits
+    index = S.SamIndex(corpus, [cfgs[0].separator])
+    want, got, errors = [None, None], [None, None], []
+    inputs = []
+    for cfg in cfgs:
+        scripts = W.make_scripts(cfg, corpus)
+        noise = W.make_noise_logits(cfg)
+        rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+        inputs.append((scripts, noise, rowmax))
+    for i, cfg in enumerate(cfgs):
+        scripts, noise, rowmax = inputs[i]
+        want[i] = W.run_closed_loop(cfg, W.ClosedLoopFeeder(cfg, scripts, rowmax),
+                                    OracleBackend(cfg, corpus, noise.copy(), oracle.host_threads()), None)
+
+    def worker(i):
+        try:
+            cfg = cfgs[i]
+            scripts, noise, rowmax = inputs[i]
+            with torch.cuda.stream(torch.cuda.Stream()):
+                be = CudaBackend(cfg, corpus, bits_to_device(noise), index=index)
+                for _ in range(3):                       # several loops per thread: more chances to collide
+                    be.state.zero_(); be.mlen.zero_()
+                    got[i] = W.run_closed_loop(cfg, W.ClosedLoopFeeder(cfg, scripts, rowmax), be, None)
+                    assert be.status() == 0
+                    _assert_traces_equal(want[i], got[i])
+        except BaseException as e:                       # reported by the main thread
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
