@@ -431,7 +431,7 @@ constexpr int kTileVec = 1024;    // 16-byte vectors per tile: 16 KB
 constexpr int kVecPerThread = kTileVec / kArgmaxThreads;
 
 // Turn a thread's (best value, vector index) into a packed candidate by re-reading that one
-// vector (an L2 hit: it was streamed moments ago) and locating the first equal element.
+// vector and locating the first equal element.
 __device__ __forceinline__ unsigned long long resolve_candidate(const RowView& rv, int V, float best, int bestq,
                                                                 int v_offset) {
     if (bestq < 0) return 0ull;
@@ -472,7 +472,14 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
 
     auto flush = [&]() {
         if (cur_row < 0) return;
-        unsigned long long k = first_nan ? kCandidateFirstIsNaN : resolve_candidate(rv, V, best, bestq, rm.v_offset);
+        // Only a lane that holds the warp's largest value can win, so only those lanes go back to memory for
+        // the position of their element (usually one lane; every lane doing so re-read 8 % of the logits).
+        float wbest = best;                         // never NaN: only values greater than -inf are kept
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) wbest = fmaxf(wbest, __shfl_xor_sync(kFull, wbest, d));
+        unsigned long long k = 0ull;
+        if (first_nan) k = kCandidateFirstIsNaN;
+        else if (best == wbest) k = resolve_candidate(rv, V, best, bestq, rm.v_offset);
         k = warp_max_u64(k);
         if (lane == 0 && k != 0ull) atomicMax(keys + cur_row, k);
     };
