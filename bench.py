@@ -37,6 +37,11 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
 # capture summarised in profiles/launch_list_cfg2.md (config 2, argmax_bulk_kernel; traffic scales with rows)
 NCU_DRAM_BYTES_PER_ROW = 304325.1
+# the same for argmax_direct_kernel (--variant 1; profiles/argmax_direct_kernel_cfg2_launch_list.md); that capture was
+# taken at V = 151,936, and the figure is only reported for that row length
+NCU_DRAM_BYTES_PER_ROW_DIRECT = 304501.7
+# and for the same kernel on the paper's evaluation shape (config 5: 16 rows per launch)
+NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE = 305006.6
 # dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
 NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 46.9
 
@@ -382,6 +387,13 @@ def run_ours(args):
         kernel_ms, kernel_name = total_ms / args.steps, "argmax_bulk_kernel (argmax + fused accept/walk/draft tail)"
     else:
         kernel_ms, kernel_name = (split["argmax_ms"] if split else total_ms / args.steps), "argmax kernel alone"
+    # counters exist for the two kernels at the full vocabulary; the latency case (short proposals over little data)
+    # runs the direct-load kernel whatever the variant
+    latency_case = args.variant == 0 and cfg.K <= 4 and R * cfg.vocab * 2 <= (96 << 20)
+    traffic_per_row = None
+    if cfg.vocab == 151936:
+        traffic_per_row = (NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE if latency_case else
+                           NCU_DRAM_BYTES_PER_ROW_DIRECT if args.variant == 1 else NCU_DRAM_BYTES_PER_ROW)
     achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
     walk = None
     if split is not None:
@@ -414,7 +426,7 @@ def run_ours(args):
         "launches_per_step": launches_per_step, "variant": args.variant, "cuda_graph": bool(args.graph), "back_to_back": back_to_back,
         "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
-                     "traffic": (NCU_DRAM_BYTES_PER_ROW * (rows_read_per_step if args.skip_unused_rows else R)) if NCU_DRAM_BYTES_PER_ROW else None,
+                     "traffic": traffic_per_row * (rows_read_per_step if args.skip_unused_rows else R) if traffic_per_row else None,
                      "algorithmic_bytes": alg_bytes,
                      "whole_step": {"ms": total_ms / args.steps, "achieved": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9,
                                     "frac": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9 / peak,
