@@ -178,7 +178,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         const int64_t nvec_max = (static_cast<int64_t>(V) + 7 + 7) / 8;   // worst-case leading offset of 7 elements
         const int tiles_per_row = static_cast<int>((nvec_max + kTileVec - 1) / kTileVec);
         const int64_t total = R * tiles_per_row;
-        int64_t grid = static_cast<int64_t>(di.sms) * 4;
+        int64_t grid = static_cast<int64_t>(di.sms) * kDirectCtasPerSm;
         if (grid > total) grid = total;
         if (grid < 1) grid = 1;
         argmax_direct_kernel<<<static_cast<unsigned>(grid), kArgmaxThreads, 0, st>>>(
