@@ -196,7 +196,7 @@ int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st, bo
     const unsigned grid = static_cast<unsigned>((a.B + warps - 1) / warps);
     if (!after_own_argmax) {
         // whatever precedes in the stream may still be producing this kernel's inputs: ordinary stream order
-        accept_kernel<kMode><<<grid, warps * 32, 0, st>>>(sam, a);
+        accept_kernel<kMode, false><<<grid, warps * 32, 0, st>>>(sam, a);
         SAM_CUDA(cudaGetLastError());
         ++g_launches;
         return SAM_OK;
@@ -213,7 +213,7 @@ int launch_accept(const DeviceSam& sam, const AcceptArgs& a, cudaStream_t st, bo
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    SAM_CUDA(cudaLaunchKernelEx(&cfg, accept_kernel<kMode>, sam, a));
+    SAM_CUDA(cudaLaunchKernelEx(&cfg, accept_kernel<kMode, true>, sam, a));
     ++g_launches;
     return SAM_OK;
 }

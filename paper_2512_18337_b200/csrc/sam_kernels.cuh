@@ -575,8 +575,19 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
     }
     const int nd = (p.flags & kNoSpeculation) ? 0 : max(0, min(p.n_draft[b], K));
     const int d = (lane < K) ? p.drafts[static_cast<long long>(b) * K + lane] : -1;
+    RecRegs rj = root_rec();     // lane j: record of the state reached after j + 1 drafts
+    // Launched as a dependent of the argmax kernel and with no walk-ahead done there: the time until that grid has
+    // finished is used to follow the whole proposal here, lane j keeping what was reached after j + 1 drafts.
+    constexpr bool kWalkBeforeWait = kMode == kTailFullWalk && kAfterGrid;
+    if (kWalkBeforeWait) {
+        int s2 = s, L2 = L;
+        RecRegs r2 = r;
+        for (int j = 0; j < nd; ++j) {
+            walk_token(sam, __shfl_sync(kFull, d, j), s2, L2, r2, lane);
+            if (lane == j) { ps = s2; pl = L2; rj = r2; }
+        }
+    }
     if (kAfterGrid) asm volatile("griddepcontrol.wait;" ::: "memory");
-    RecRegs rj = root_rec();     // kTailResume: lane j fetches the record of the state reached after j + 1 drafts
     if (kMode == kTailResume && lane < nd) {
         ps = __ldcg(p.pre_state + static_cast<long long>(b) * K + lane);
         pl = __ldcg(p.pre_len + static_cast<long long>(b) * K + lane);
@@ -626,7 +637,7 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
     }
 
     if (kMode != kTailVerifyOnly) {
-        if (kMode == kTailResume) {
+        if (kMode == kTailResume || kWalkBeforeWait) {
             // the walk over the accepted draft prefix was done ahead of time
             if (a > 0) {
                 const int src = a - 1;
@@ -658,13 +669,15 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
     }
 }
 
-template <int kMode>
+// kDependent: launched as a programmatic dependent of the argmax kernel (waits for that grid inside);
+// otherwise an ordinary launch behind whatever produced the row results.
+template <int kMode, bool kDependent = true>
 __global__ void __launch_bounds__(128)
 accept_kernel(DeviceSam sam, AcceptArgs p) {
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= p.B) return;
-    accept_stream<kMode, true>(sam, p, b, lane);
+    accept_stream<kMode, kDependent>(sam, p, b, lane);
 }
 
 __global__ void __launch_bounds__(32 * kMaxSlots)
