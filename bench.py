@@ -40,7 +40,7 @@ NCU_DRAM_BYTES_PER_ROW = 304325.1
 # the same for argmax_direct_kernel (--variant 1; profiles/argmax_direct_kernel_cfg2_launch_list.md); that capture was
 # taken at V = 151,936, and the figure is only reported for that row length
 NCU_DRAM_BYTES_PER_ROW_DIRECT = 304681.8
-# and for the same kernel on the paper's evaluation shape (config 5: 16 rows per launch)
+# and for the same kernel on the paper's evaluation shape (config 5: 16 rows per launch; used for workloads that fit in L2)
 NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE = 305045.6
 # dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
 NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 46.9
@@ -259,7 +259,7 @@ def run_ours(args):
     # of its own, so that the library's events separate the vocabulary argmax from accept + walk + draft
     split = None
     if args.split_steps > 0:
-        S.sam_set_argmax_variant(0 if args.variant == 2 else args.variant)
+        S.sam_set_argmax_variant(3 if args.variant == 2 else args.variant)
         S.sam_profile_enable(args.split_steps)
         n_before = len(stats_trace)
         for i in range(args.split_steps):
@@ -387,13 +387,14 @@ def run_ours(args):
         kernel_ms, kernel_name = total_ms / args.steps, "argmax_bulk_kernel (argmax + fused accept/walk/draft tail)"
     else:
         kernel_ms, kernel_name = (split["argmax_ms"] if split else total_ms / args.steps), "argmax kernel alone"
-    # counters exist for the two kernels at the full vocabulary; the latency case (short proposals over little data)
-    # runs the direct-load kernel whatever the variant
-    latency_case = args.variant == 0 and cfg.K <= 4 and R * cfg.vocab * 2 <= (96 << 20)
+    # counters exist for the two argmax kernels at the full vocabulary
+    # the library's own rule for variant 0: direct loads up to 768 MiB of logits and K <= 16
+    direct = args.variant == 1 or (args.variant == 0 and cfg.K <= 16 and R * cfg.vocab * 2 <= (768 << 20))
     traffic_per_row = None
     if cfg.vocab == 151936:
-        traffic_per_row = (NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE if latency_case else
-                           NCU_DRAM_BYTES_PER_ROW_DIRECT if args.variant == 1 else NCU_DRAM_BYTES_PER_ROW)
+        traffic_per_row = (NCU_DRAM_BYTES_PER_ROW if not direct else
+                           NCU_DRAM_BYTES_PER_ROW_DIRECT if R * cfg.vocab * 2 > (126 << 20) else
+                           NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE)
     achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
     walk = None
     if split is not None:
@@ -424,7 +425,7 @@ def run_ours(args):
         "stream_steps_per_s": world * cfg.B * args.steps / (max_ms / 1e3),
         "gpu_launches": launches,
         "launches_per_step": launches_per_step, "variant": args.variant, "cuda_graph": bool(args.graph), "back_to_back": back_to_back,
-        "roofline": {"kernel": kernel_name, "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": kernel_name + (" (argmax_direct_kernel)" if direct else " (argmax_bulk_kernel)" if launches_per_step != 1 else ""), "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
                      "traffic": traffic_per_row * (rows_read_per_step if args.skip_unused_rows else R) if traffic_per_row else None,
                      "algorithmic_bytes": alg_bytes,
@@ -808,9 +809,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--presleep-cycles", type=int, default=300000,
                     help="length of the spin kernel enqueued before each timed step (outside the events)")
-    ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 2],
-                    help="kernel selection of the library (0 = default: bulk-copy argmax kernel + accept kernel; "
-                         "1 = direct-load argmax + accept; 2 = one kernel per step with the accept step inside)")
+    ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="kernel selection of the library (0 = default: by size - bulk-copy argmax kernel above 768 MiB of "
+                         "logits or K > 16, direct-load kernel below, each + accept kernel; 1 = direct-load argmax + accept; "
+                         "2 = bulk-copy kernel with the accept step inside, one launch per step; 3 = bulk-copy + accept)")
     ap.add_argument("--split-steps", type=int, default=50,
                     help="steps run after the timed region with two kernels per step, to report each kernel's time")
     ap.add_argument("--cpu-steps", type=int, default=200)

@@ -404,11 +404,15 @@ int sam_multi_step(const sam_set* set,
  * Process-wide state, not thread-safe; enable/disable is not a hot-path call. */
 int sam_profile_enable(int32_t max_calls);
 /* Selects the kernels of sam_verify / sam_step for later calls (process-wide; for measurements
- * and tests): 0 = automatic (default: a bulk-copy pipelined argmax kernel when the logits base
- * and row stride are 16-byte aligned, a direct-load kernel otherwise or when K <= 4 and the logits
- * are under 96 MiB, each followed by the accept kernel), 1 = always direct loads, 2 = as 0, but the bulk-copy kernel also runs the accept step of
- * every stream as soon as its rows are complete (one launch per call; measured slightly slower than
- * two launches on B200), 3 = same as 0. */
+ * and tests):
+ *   0 = automatic (default): the bulk-copy pipelined argmax kernel when the logits base and row
+ *       stride are 16-byte aligned and the call is large (more than 768 MiB of logits, or K > 16);
+ *       the direct-load kernel otherwise; each followed by the accept kernel as a dependent launch;
+ *   1 = always the direct-load kernel;
+ *   2 = the bulk-copy kernel whenever the rows are aligned, with the accept step of every stream
+ *       inside it, run as soon as the stream's rows are complete (one launch per call; measured
+ *       slightly slower than two launches on B200);
+ *   3 = the bulk-copy kernel whenever the rows are aligned, followed by the accept kernel. */
 int sam_set_argmax_variant(int32_t variant);
 int32_t sam_profile_count(void);
 int sam_profile_read(int32_t call, float* argmax_ms, float* accept_ms);

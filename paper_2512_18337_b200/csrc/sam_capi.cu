@@ -79,7 +79,7 @@ int check_verify_args(const void* logits, int64_t stride, int32_t B, int32_t K, 
     return SAM_OK;
 }
 
-int g_argmax_variant = 0;   // 0/3 = choose by alignment, 1 = direct loads always, 2 = as 0 with the accept step inside the argmax kernel
+int g_argmax_variant = 0;   // 0 = by alignment and size, 1 = direct loads always, 2 = bulk-copy (if aligned) with the accept step inside, 3 = bulk-copy (if aligned) + accept kernel
 
 inline int* status_word(unsigned long long* keys, int64_t R) {
     return reinterpret_cast<int*>(reinterpret_cast<char*>(keys) + ((R * 8 + 255) / 256) * 256);
@@ -124,11 +124,14 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
                   int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
                   bool* did_prewalk = nullptr, const AcceptArgs* tail = nullptr, int tail_mode = 0,
                   int* done = nullptr, bool* did_tail = nullptr, const RowMap* rmap = nullptr) {
-    // Short proposals over little data (the paper's own setting: batch 4, three speculative tokens) are a latency
-    // case: the direct-load kernel starts faster than the bulk-copy pipeline and there is little for a walk-ahead to
-    // save (measured at K = 3: 12.2 vs 13.4 us per step for 4 streams, 25.2 vs 26.5 us for 64; equal near 200 MB of logits).
-    const bool latency_case = g_argmax_variant == 0 && tail != nullptr && tail->K <= 4 &&
-                              R * static_cast<int64_t>(V) * 2 <= (int64_t(96) << 20);
+    // Below about 0.8 GB of logits the direct-load kernel followed by an accept kernel that walks the proposal before its
+    // grid-dependency wait is the faster pair: it starts sooner than the bulk-copy pipeline and finishes more evenly
+    // (measured per step, direct vs bulk-copy: 11.4 vs 13.4 us at B = 4, K = 3; 11.7 vs 13.8 us on the tiny workload;
+    // 39.2 vs 40.9 us at 175 MB; 105.9 vs 107.1 us at 660 MB; 153.2 vs 151.2 us at 990 MB; 197.1 vs 195.3 us at 1.3 GB).
+    // Proposals longer than 16 tokens stay with the bulk-copy kernel at every size: their walk-ahead is long and its
+    // spare warps hide it better (K = 32: 45.6 vs 38.2 us at 160 MB).
+    const bool latency_case = g_argmax_variant == 0 && tail != nullptr && tail->K <= 16 &&
+                              R * static_cast<int64_t>(V) * 2 <= (int64_t(768) << 20);
     prof_mark(0, st);
     DeviceInfo di;
     int rc = device_info(&di);

@@ -66,7 +66,7 @@ def test_verify_random_shapes_and_values(seed):
     ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
     S.sam_workspace_init(ws, wsb)
     d, nd_t = _i32(drafts), _i32(n_draft)
-    for variant in (0, 1, 2):
+    for variant in (0, 1, 2, 3):
         am = torch.full((B, K + 1), -9, dtype=torch.int32, device=DEV)
         acc = torch.full((B, K + 1), -9, dtype=torch.int32, device=DEV)
         nacc = torch.full((B,), -9, dtype=torch.int32, device=DEV)
@@ -83,7 +83,7 @@ def test_verify_random_shapes_and_values(seed):
 
 @pytest.mark.parametrize("vocab,K,mm,variant", [
     (2, 4, 1, 0), (3, 32, 2, 0), (5, 8, 3, 1), (17, 16, 2, 0),
-    (8, 8, 2, 0), (8, 8, 2, 2), (16, 32, 1, 0), (24, 5, 4, 2), (32, 16, 2, 0),
+    (8, 8, 2, 3), (8, 8, 2, 2), (16, 32, 1, 0), (24, 5, 4, 2), (32, 16, 2, 3),
 ])
 def test_closed_loop_small_alphabets(vocab, K, mm, variant):
     """Two to thirty-two distinct tokens: long runs, clones everywhere, suffix-link chains dozens deep.

@@ -23,6 +23,8 @@ pytestmark = pytest.mark.gpu
     ("tiny", 0, 0),
     ("cfg2_small", 0, 0),
     ("cfg2_small", 2, 0),
+    ("cfg2_small", 3, 0),
+    ("cfg2_small", 3, S.SAM_STEP_SKIP_UNUSED_ROWS),
     ("cfg2_small", 0, S.SAM_STEP_SKIP_UNUSED_ROWS),
     ("paper_shape", 0, 0),
 ])

@@ -24,7 +24,7 @@ def _i32(x):
 
 @pytest.mark.parametrize("V,pad,B,K", [(1000, 0, 5, 8), (4097, 3, 7, 4), (151936, 0, 3, 16), (151936, 8, 40, 2),
                                        (8192 * 13 + 24, 0, 9, 5), (7, 0, 300, 1), (65536, 0, 2, 32)])
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", [0, 1, 3])
 def test_verify_skipping_unused_rows(V, pad, B, K, variant):
     rng = np.random.default_rng(V + B + K)
     R = B * (K + 1)
@@ -61,7 +61,7 @@ def test_verify_skipping_unused_rows(V, pad, B, K, variant):
     assert S.sam_workspace_status(ws, B, K) == 0
 
 
-@pytest.mark.parametrize("variant,skip", [(0, True), (0, False), (1, True), (2, False)])
+@pytest.mark.parametrize("variant,skip", [(0, True), (0, False), (1, True), (2, False), (3, True), (3, False)])
 def test_closed_loop_with_the_adaptive_switch(variant, skip):
     """A schedule of context lengths drives the switch: steps over the threshold run without speculation.
     Every output of every step and the final counters equal the oracle's."""

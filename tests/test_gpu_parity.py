@@ -53,9 +53,10 @@ def _check_verify(bits, V, B, K, rng):
         keep = rng.random(nd) < 0.8
         drafts[b, :nd] = np.where(keep, am_o[b, :nd], rng.integers(0, V, size=nd))
     acc_o, nacc_o = oracle.accept_batch(drafts, n_draft, am_o)
-    # 0: bulk-copy pipeline (when rows are 16-byte aligned) followed by the accept kernel;
-    # 1: direct loads always; 2: bulk-copy pipeline with the accept step inside the same kernel
-    for variant in (0, 1, 2):
+    # 0: chosen by alignment and size (these small cases: direct loads); 1: direct loads always;
+    # 2: bulk-copy pipeline (when rows are 16-byte aligned) with the accept step inside the same kernel;
+    # 3: bulk-copy pipeline followed by the accept kernel
+    for variant in (0, 1, 2, 3):
         am, acc, nacc = _verify_gpu(bits, V, B, K, drafts, n_draft, variant=variant)
         assert (am == am_o).all(), variant
         assert (nacc == nacc_o).all() and (acc == acc_o).all(), variant
@@ -282,7 +283,7 @@ def test_closed_loop_cfg1_full():
     _assert_traces_equal(tr_o, tr_g)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_closed_loop_other_kernel_variants(variant):
     """The step with direct loads (full walk in the accept kernel) and with the accept step inside the
     bulk-copy argmax kernel gives the same trace as the oracle."""
