@@ -1,4 +1,4 @@
-"""Closed-loop parity at the full sizes of the three large workloads, tolerance 0.
+"""Closed-loop parity at the full sizes of the three large workloads and of the paper's own evaluation shape, tolerance 0.
 
 Same launch configuration as the benchmark (every stream, full vocabulary, the full corpus, the
 fused step).  The noise logits are drawn once on the device and copied to the host, so the CPU
@@ -59,3 +59,8 @@ def test_full_size_cfg3_verify_heavy_with_ties():
 def test_full_size_cfg4_long_trace():
     """B=1024, K=32 (the largest draft length), min_match=4, 64M-token corpus, 10.3 GB of logits per step."""
     _full_size_closed_loop(4, steps=3)
+
+
+def test_full_size_cfg5_paper_evaluation_shape():
+    """B=4, K=3 (one autoregressive + three speculative tokens per step), 1M-token corpus, all 64 steps."""
+    _full_size_closed_loop(5, steps=64)
