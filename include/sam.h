@@ -321,6 +321,9 @@ int sam_pending(sam_index* idx, int64_t* tokens_queued, int64_t* tokens_built, i
  * copied instead after the wide-edge area had to be laid out afresh).  Does not wait for the
  * builder thread and does not synchronise the stream; hot-path calls enqueued afterwards on the
  * same stream see the grown automaton.  Call it from the thread that makes the hot-path calls.
+ * The first small update creates 1 MiB of page-locked host memory and an event for the handle
+ * (released by sam_free); a later call may wait on the host until the previous update's copy has
+ * left that buffer.
  * After it, run sam_renormalize on every batch of stream states that will be used again.
  * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_TOO_LARGE (the automaton no longer
  * fits the blob), SAM_ERR_CUDA. */

@@ -1,6 +1,7 @@
 // C ABI of the library: argument checks, device-blob upload and kernel launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 #include <cstdlib>
 #include <atomic>
@@ -259,9 +260,80 @@ int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st) {
     StateRec* rec = reinterpret_cast<StateRec*>(base + L.rec_off);
     Edge* wide = reinterpret_cast<Edge*>(base + L.edge_off);
     int32_t* root = reinterpret_cast<int32_t*>(base + L.root_off);
+    const int64_t n_rec = static_cast<int64_t>(D.rec_ids.size());
+    // ---- small update (the usual case between two decoding steps): everything but rows long enough to be copied
+    // on their own goes through one page-locked buffer, one copy and one kernel
+    {
+        constexpr int64_t kPinnedBytes = int64_t(1) << 20;
+        auto up32 = [](int64_t x) { return (x + 31) & ~int64_t(31); };
+        int64_t n_seg = 0, n_edges = 0;
+        for (const WideSeg& g : D.segs)
+            if (g.len < kDirectRowEdges) { ++n_seg; n_edges += g.len; }
+        const int64_t n_root = static_cast<int64_t>(D.root_tok.size());
+        const int64_t n_tail = static_cast<int64_t>(D.corpus_tail.size());
+        UpdateArgs a{};
+        a.off_ids = 0;
+        a.off_recs = up32(n_rec * 4);
+        a.off_descs = a.off_recs + n_rec * static_cast<int64_t>(sizeof(StateRec));
+        a.off_edges = up32(a.off_descs + n_seg * static_cast<int64_t>(sizeof(SegDesc)));
+        a.off_rtok = up32(a.off_edges + n_edges * static_cast<int64_t>(sizeof(Edge)));
+        a.off_rdst = up32(a.off_rtok + n_root * 4);
+        a.off_tail = up32(a.off_rdst + n_root * 4);
+        const int64_t total = up32(a.off_tail + n_tail * 4);
+        if (total <= kPinnedBytes && total <= L.stage_bytes) {
+            if (!idx->pinned_stage) {
+                void* hp = nullptr;
+                cudaEvent_t ev = nullptr;
+                SAM_CUDA(cudaHostAlloc(&hp, static_cast<size_t>(kPinnedBytes), cudaHostAllocDefault));
+                const cudaError_t e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+                if (e != cudaSuccess) { cudaFreeHost(hp); return cuda_fail(e); }
+                idx->pinned_stage = hp;
+                idx->pinned_bytes = kPinnedBytes;
+                idx->stage_event = ev;
+            } else {
+                // the previous update's copy must have left the buffer before it is refilled
+                SAM_CUDA(cudaEventSynchronize(static_cast<cudaEvent_t>(idx->stage_event)));
+            }
+            char* h = static_cast<char*>(idx->pinned_stage);
+            std::memcpy(h + a.off_ids, D.rec_ids.data(), static_cast<size_t>(n_rec) * 4);
+            std::memcpy(h + a.off_recs, D.recs.data(), static_cast<size_t>(n_rec) * sizeof(StateRec));
+            SegDesc* descs = reinterpret_cast<SegDesc*>(h + a.off_descs);
+            Edge* edges = reinterpret_cast<Edge*>(h + a.off_edges);
+            int64_t ns = 0, ne = 0;
+            for (const WideSeg& g : D.segs) {
+                if (g.len >= kDirectRowEdges) continue;
+                descs[ns++] = SegDesc{g.dst_off, static_cast<int>(ne), g.len};
+                std::memcpy(edges + ne, D.seg_edges.data() + g.src_off, static_cast<size_t>(g.len) * sizeof(Edge));
+                ne += g.len;
+            }
+            std::memcpy(h + a.off_rtok, D.root_tok.data(), static_cast<size_t>(n_root) * 4);
+            std::memcpy(h + a.off_rdst, D.root_dst.data(), static_cast<size_t>(n_root) * 4);
+            std::memcpy(h + a.off_tail, D.corpus_tail.data(), static_cast<size_t>(n_tail) * 4);
+            if (total > 0) {
+                SAM_CUDA(cudaMemcpyAsync(stage, h, static_cast<size_t>(total), cudaMemcpyHostToDevice, st));
+                SAM_CUDA(cudaEventRecord(static_cast<cudaEvent_t>(idx->stage_event), st));
+                a.rec = rec; a.wide = wide; a.root = root;
+                a.corpus = reinterpret_cast<int32_t*>(base + L.corpus_off) + D.corpus_off;
+                a.stage = stage;
+                a.n_rec = static_cast<int>(n_rec); a.n_seg = static_cast<int>(n_seg);
+                a.n_root = static_cast<int>(n_root); a.n_tail = static_cast<int>(n_tail);
+                a.root_span = static_cast<int>(L.root_span);
+                const int64_t work = std::max(std::max(n_rec, n_seg * 32), std::max(n_root, n_tail));
+                const unsigned blocks = static_cast<unsigned>(std::min<int64_t>(1184, std::max<int64_t>(1, (work + 255) / 256)));
+                apply_update_kernel<<<blocks, 256, 0, st>>>(a);
+                SAM_CUDA(cudaGetLastError());
+                ++g_launches;
+            }
+            for (const WideSeg& g : D.segs)
+                if (g.len >= kDirectRowEdges)
+                    SAM_CUDA(cudaMemcpyAsync(wide + g.dst_off, D.seg_edges.data() + g.src_off,
+                                             static_cast<size_t>(g.len) * sizeof(Edge), cudaMemcpyHostToDevice, st));
+            return SAM_OK;
+        }
+    }
+    // ---- large update: section by section through the staging area
     std::vector<char> buf;
     // records: [ids (padded to 32 B)] [records]
-    const int64_t n_rec = static_cast<int64_t>(D.rec_ids.size());
     const int64_t per_round = (L.stage_bytes - 64) / 36;
     for (int64_t i0 = 0; i0 < n_rec; i0 += per_round) {
         const int64_t n = std::min(per_round, n_rec - i0);
@@ -458,6 +530,11 @@ int sam_upload(sam_index* idx, void* device_buf, int64_t bytes, void* cuda_strea
 
 void sam_free(sam_index* idx) {
     if (!idx) return;
+    if (idx->stage_event) {
+        cudaEventSynchronize(static_cast<cudaEvent_t>(idx->stage_event));
+        cudaEventDestroy(static_cast<cudaEvent_t>(idx->stage_event));
+    }
+    if (idx->pinned_stage) cudaFreeHost(idx->pinned_stage);
     dyn_destroy(idx);
     delete idx;
 }

@@ -108,6 +108,11 @@ struct sam_index {
     // growing index only
     samb200::DynIndex* dyn = nullptr;
     int64_t updates_incremental = 0, updates_full = 0, update_bytes = 0;   // what sam_sync has applied so far
+    // page-locked staging for small updates and the event that says when its last copy has left it (CUDA objects,
+    // created by the first incremental update, released by sam_free)
+    void* pinned_stage = nullptr;
+    int64_t pinned_bytes = 0;
+    void* stage_event = nullptr;
 };
 
 namespace samb200 {

@@ -53,6 +53,51 @@ scatter_root_kernel(int32_t* __restrict__ root_dst, const int32_t* __restrict__ 
     if (t >= 0 && t < span) root_dst[t] = dst[i];
 }
 
+// A whole small update in one launch: the staged buffer holds record ids and records, row descriptors and
+// their edges, root entries and the appended text; every destination is written by exactly one thread (records,
+// root entries, text) or one warp (rows), and the four parts touch different arrays.
+struct UpdateArgs {
+    StateRec* rec;
+    Edge* wide;
+    int32_t* root;
+    int32_t* corpus;        // where the appended text goes
+    const char* stage;
+    long long off_ids, off_recs, off_descs, off_edges, off_rtok, off_rdst, off_tail;
+    int n_rec, n_seg, n_root, n_tail, root_span;
+};
+
+__global__ void __launch_bounds__(256)
+apply_update_kernel(UpdateArgs a) {
+    const int nthreads = gridDim.x * blockDim.x;
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int32_t* ids = reinterpret_cast<const int32_t*>(a.stage + a.off_ids);
+    const StateRec* recs = reinterpret_cast<const StateRec*>(a.stage + a.off_recs);
+    for (int i = gtid; i < a.n_rec; i += nthreads) {
+        const int4* src = reinterpret_cast<const int4*>(recs + i);
+        int4* dst = reinterpret_cast<int4*>(a.rec + ids[i]);
+        const int4 x = src[0], y = src[1];
+        dst[0] = x;
+        dst[1] = y;
+    }
+    const SegDesc* segs = reinterpret_cast<const SegDesc*>(a.stage + a.off_descs);
+    const Edge* staged = reinterpret_cast<const Edge*>(a.stage + a.off_edges);
+    for (int w = gtid >> 5; w < a.n_seg; w += nthreads >> 5) {
+        const SegDesc g = segs[w];
+        const int2* src = reinterpret_cast<const int2*>(staged + g.src_off);
+        int2* dst = reinterpret_cast<int2*>(a.wide + g.dst_off);
+        for (int k = lane; k < g.len; k += 32) dst[k] = src[k];
+    }
+    const int32_t* rtok = reinterpret_cast<const int32_t*>(a.stage + a.off_rtok);
+    const int32_t* rdst = reinterpret_cast<const int32_t*>(a.stage + a.off_rdst);
+    for (int i = gtid; i < a.n_root; i += nthreads) {
+        const int t = rtok[i];
+        if (t >= 0 && t < a.root_span) a.root[t] = rdst[i];
+    }
+    const int32_t* tail = reinterpret_cast<const int32_t*>(a.stage + a.off_tail);
+    for (int i = gtid; i < a.n_tail; i += nthreads) a.corpus[i] = tail[i];
+}
+
 // After the text has grown, a stream's string of length L may belong to a state that was split off
 // its old one: the state of a string is the one with len(link(s)) < L <= len(s).  Climb suffix links
 // until that holds.  One thread per stream.

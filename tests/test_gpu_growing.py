@@ -179,3 +179,44 @@ def test_builder_thread_and_empty_start():
     st.zero_(); ml.zero_()
     _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm)
     assert (ml_o == ld).all()
+
+
+def test_small_and_large_updates_take_their_own_paths():
+    """Updates of a few hundred tokens go through one page-locked buffer, one copy and one kernel; an update of
+    tens of thousands of tokens is too large for that buffer and is applied section by section.  Both leave the
+    device copy equal to the oracle's automaton (drafts, states and matched lengths of streams that read all over
+    the grown text), whichever order they come in."""
+    rng = np.random.default_rng(11)
+    sep, K, mm, B, ld = 1000, 6, 2, 64, 12
+    text = _hub_text(rng, 2000, sep)
+    index = S.SamIndex(text, [sep], max_tokens=120000, max_token_id=sep + 50)
+    osam = oracle.OracleSAM(text, [sep])
+    st = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ml = torch.zeros(B, dtype=torch.int32, device=DEV)
+    st_o = np.zeros(B, np.int32)
+    ml_o = np.zeros(B, np.int32)
+    sizes = [300, 40000, 150, 25000, 60, 1]
+    for rnd, n in enumerate(sizes):
+        piece = _hub_text(rng, n, sep)
+        osam.extend(piece)
+        inc0, full0, bytes0 = S.sam_update_stats(index.handle)
+        S.sam_extend(index.handle, piece)
+        assert S.sam_sync(index.handle) == osam.n
+        inc1, full1, bytes1 = S.sam_update_stats(index.handle)
+        assert inc1 + full1 > inc0 + full0
+        if n >= 25000:
+            assert bytes1 - bytes0 > (1 << 20)          # more than the page-locked buffer holds
+        elif full1 == full0:
+            assert bytes1 - bytes0 < (1 << 20)
+        osam.renormalize(st_o, ml_o)
+        S.sam_renormalize(index.handle, B, st, ml)
+        toks = np.empty((B, ld), np.int32)
+        for b in range(B):
+            start = int(rng.integers(0, osam.n - ld))
+            toks[b] = osam.corpus[start:start + ld]
+        toks[rng.random((B, ld)) < 0.05] = sep + 7
+        n_new = rng.integers(0, ld + 1, size=B).astype(np.int32)
+        _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm)
+    ex, oe = S.sam_export(index.handle), osam.export()
+    for k in oe:
+        assert (ex[k] == oe[k]).all(), k
