@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_DRAM_BYTES_PER_ROW = 304325.1
 # the same for argmax_direct_kernel (--variant 1; profiles/argmax_direct_kernel_cfg2_launch_list.md); that capture was
 # taken at V = 151,936, and the figure is only reported for that row length
-NCU_DRAM_BYTES_PER_ROW_DIRECT = 304681.8
+NCU_DRAM_BYTES_PER_ROW_DIRECT = 304694.3
 # and for the same kernel on the paper's evaluation shape (config 5: 16 rows per launch; used for workloads that fit in L2)
 NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE = 305051.8
 # dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
