@@ -184,6 +184,10 @@ def test_argument_checks_that_need_no_device():
     finally:
         S.sam_free(h)
     assert S.sam_strerror(-3).startswith("automaton not uploaded")
+    # the kernel-selection switch takes 0..3 and keeps its value on a refused call
+    for v in (1, 2, 3, 0):
+        assert lib.sam_set_argmax_variant(v) == 0
+    assert lib.sam_set_argmax_variant(4) == -1 and lib.sam_set_argmax_variant(-1) == -1
 
 
 def test_missing_library_fails_loudly(tmp_path):
