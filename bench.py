@@ -8,6 +8,11 @@ over [B, K+1, V] bf16 logits, prefix accept, automaton walk over the accepted to
 (`sam_step`).  The workload is synthetic (see workload/agent_memory.py); the default is the
 B=256, K=16, 16M-token-corpus configuration.  Prints ONE JSON line on rank 0.
 
+`--gpus N` with N > 1 starts N ranks, one per GPU (it re-runs itself under
+`python -m torch.distributed.run`; started under such a launcher already, it checks that the world size
+is N).  Every rank owns B streams of its own and a replica of the index; no collective touches the data
+path, the ranks only meet for the final sum of tokens and maximum of time (weak scaling).
+
 Timing: every step is bracketed by CUDA events on the launching stream; the stand-in target
 model (sparse planting of the wanted tokens into the resident noise logits between steps) is
 outside the events.  `--impl reference` times the CPU oracle instead (host cores, wall clock).
@@ -48,7 +53,80 @@ NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 46.9
 
 # ----------------------------------------------------------------------------- helpers
 def dist_env():
-    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+    from harness.launcher import rank_env
+    return rank_env()
+
+
+RANK_SEED_STRIDE = 7919      # rank r draws its stream scripts and planting decisions from seed + 7919 * r
+
+
+def plan_rank(args, rank: int):
+    """(cfg, stream_cfg) of one rank.  cfg describes what every rank shares (corpus, noise logits, sizes);
+    stream_cfg differs only in the seed of the B streams the rank owns."""
+    base = W.CONFIGS[args.config]
+    if args.streams > 0:
+        base = base.scaled(B=args.streams, name=f"{base.name}_B{args.streams}")
+    # long enough for every leg of either arm (the oracle leg replays the scripts from step 0), and the same in
+    # both arms: the script generator's draws depend on the script length
+    n_script_steps = max(args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1, args.cpu_steps + 8)
+    cfg = base.scaled(steps=n_script_steps)
+    stream_cfg = cfg.scaled(seed=cfg.seed + RANK_SEED_STRIDE * rank) if rank > 0 else cfg
+    return cfg, stream_cfg
+
+
+def init_ranks(backend: str, args, device_of=None):
+    """Joins the process group when started under a launcher; (rank, local_rank, world).  Refuses to run when
+    the launcher's world size is not the --gpus that was asked for."""
+    rank, local_rank, world = dist_env()
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if world > 1:
+        import torch.distributed as dist
+        kw = {}
+        if device_of is not None:
+            kw["device_id"] = device_of(local_rank)
+        dist.init_process_group(backend, **kw)
+    return rank, local_rank, world
+
+
+def gather_over_ranks(obj, world: int):
+    """List of every rank's (picklable) object, in rank order."""
+    if world == 1:
+        return [obj]
+    import torch.distributed as dist
+    out = [None] * world
+    dist.all_gather_object(out, obj)
+    return out
+
+
+NOISE_ON_HOST_MAX_BYTES = 3 << 30
+
+
+def noise_on_host(cfg) -> bool:
+    """The noise logits of both arms come from one host generator whenever that is affordable; only the
+    10 GB workload draws them on the device (minutes on the host), and its two arms then differ in bytes."""
+    return cfg.rows * cfg.vocab * 2 <= NOISE_ON_HOST_MAX_BYTES
+
+
+def workload_block(cfg) -> dict:
+    """The `config` object of the JSON line; the same for both arms."""
+    big = cfg.rows * cfg.vocab * 2 > 252e6
+    return {"workload": cfg.name, "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.vocab, "min_match": cfg.min_match,
+            "corpus_tokens": cfg.n_corpus, "accept_p": cfg.accept_p,
+            "logits_bytes_per_step": cfg.rows * cfg.vocab * 2,
+            "l2": "inputs larger than L2 (logits re-read from HBM every step)" if big
+            else "inputs smaller than 2x L2: bandwidth figures are not HBM figures",
+            "noise": "numpy PCG64 on the host, same bytes in both arms" if noise_on_host(cfg)
+            else "torch generator on the device (ours) / numpy on the host (reference): same distribution"}
+
+
+def headline(cfg, world, args, tokens, ms, **more) -> dict:
+    """The contract keys of the JSON line from the job totals (tokens summed and ms maximised over ranks)."""
+    out = {"metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic", "config": workload_block(cfg)}
+    out.update(more)
+    return out
 
 
 def reduce_over_ranks(tokens: int, ms: float, world: int, backend_device=None):
@@ -75,63 +153,109 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    """Samples SM clock, power and throttle reasons while the timed region runs: NVML from a thread of this
+    process (a sample every millisecond, so that even a 20-step window holds many), nvidia-smi as a fallback.
+    Read-only: nothing on the GPU is set."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, gpu_index: int):
-        self.lines = []
-        self.proc = None
+    def __init__(self, gpu_index: int, period_s: float = 0.001):
+        self.samples = []            # (time, sm MHz, max MHz, set of reasons)
         self.gpu = gpu_index
+        self.period = period_s
+        self.proc = None
+        self.thread = None
+        self.how = None
+        self._stop = threading.Event()
+
+    def _physical_index(self):
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [x.strip() for x in vis.split(",") if x.strip()]
+            if self.gpu < len(ids) and ids[self.gpu].isdigit():
+                return int(ids[self.gpu])
+        return self.gpu
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
-            self.thread = threading.Thread(target=self._pump, daemon=True)
+            import pynvml as N
+            N.nvmlInit()
+            h = N.nvmlDeviceGetHandleByIndex(self._physical_index())
+            mx = float(N.nvmlDeviceGetMaxClockInfo(h, N.NVML_CLOCK_SM))
+            bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+            reasons_fn = getattr(N, "nvmlDeviceGetCurrentClocksEventReasons", None) or N.nvmlDeviceGetCurrentClocksThrottleReasons
+            reasons_fn(h)       # must work before the thread relies on it
+
+            def pump():
+                while not self._stop.is_set():
+                    try:
+                        r = int(reasons_fn(h))
+                        self.samples.append((time.time(), float(N.nvmlDeviceGetClockInfo(h, N.NVML_CLOCK_SM)), mx,
+                                             {k for k, b in bits.items() if r & b}))
+                    except Exception:
+                        pass
+                    time.sleep(self.period)
+            self.thread = threading.Thread(target=pump, daemon=True)
             self.thread.start()
+            self.how = f"NVML, one sample per {self.period * 1e3:g} ms"
+            return
+        except Exception:
+            self.thread = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self._physical_index()}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "5"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
+            self.thread = threading.Thread(target=self._pump_smi, daemon=True)
+            self.thread.start()
+            self.how = "nvidia-smi -lms 5"
         except Exception:
             self.proc = None
 
-    def _pump(self):
+    def _pump_smi(self):
         for line in self.proc.stdout:
-            self.lines.append((time.time(), line.strip()))
-
-    def stop(self, t_begin: float = 0.0, t_end: float = float("inf")):
-        """Summary of the samples that arrived inside [t_begin, t_end] (the timed region)."""
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, ln in self.lines:
-            if ts < t_begin or ts > t_end:
-                continue
-            f = [x.strip() for x in ln.split(",")]
+            f = [x.strip() for x in line.strip().split(",")]
             if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
+                self.samples.append((time.time(), float(f[0]), float(f[1]),
+                                     {n for n, v in zip(self.NAMES, f[4:8]) if v.lower().startswith("active")}))
             except ValueError:
                 continue
-            for name, val in zip(names, f[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+    def stop(self, t_begin: float = 0.0, t_end: float = float("inf")):
+        """Summary of the samples that arrived inside [t_begin, t_end] (the timed region)."""
+        self._stop.set()
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no clock source available"]}
+        self.thread.join(timeout=2)
+        inside = [x for x in self.samples if t_begin <= x[0] <= t_end]
+        sm = [x[1] for x in inside]
+        reasons = set().union(*[x[3] for x in inside]) if inside else set()
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(x[2] for x in inside) if inside else None,
+                "samples": len(sm), "reasons": sorted(reasons), "source": self.how}
 
 
 def make_inputs_gpu(cfg, device):
-    """Corpus (host) and the noise logits generated on the device (seeded torch generator)."""
+    """Corpus (host) and the noise logits on the device.  The noise is drawn on the host by the generator
+    the reference arm uses and uploaded once, so both arms read the same bytes; only a workload too large
+    for that draws it on the device."""
+    import torch
     corpus = W.make_corpus(cfg)
-    logits, rowmax = W.make_noise_logits_device(cfg, device)
+    if noise_on_host(cfg):
+        bits = W.make_noise_logits(cfg)
+        rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(bits).max(axis=1))
+        logits = torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+        del bits
+    else:
+        logits, rowmax = W.make_noise_logits_device(cfg, device)
     return corpus, logits, rowmax
 
 
@@ -141,13 +265,11 @@ def run_ours(args):
     import torch.distributed as dist
     import paper_2512_18337_b200 as S
     from paper_2512_18337_b200.build import build
-    from tests.cuda_backend import CudaBackend
+    from harness.cuda_backend import CudaBackend
 
-    rank, local_rank, world = dist_env()
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    rank, local_rank, world = init_ranks("nccl", args, lambda lr: torch.device(f"cuda:{lr}"))
     device = f"cuda:{local_rank}"
     torch.cuda.set_device(device)
     if rank == 0:
@@ -156,16 +278,9 @@ def run_ours(args):
         dist.barrier()
     S.sam_set_argmax_variant(args.variant)
 
-    base = W.CONFIGS[args.config]
-    if args.streams > 0:
-        base = base.scaled(B=args.streams, name=f"{base.name}_B{args.streams}")
     # weak scaling: every rank owns B streams of its own (distinct scripts / planting draws), the
     # read-only automaton is replicated; no data-path collective
-    n_script_steps = args.warmup + args.steps + args.split_steps + 2 * args.e2e_steps + 1
-    if args.cpu_baseline and world == 1:
-        n_script_steps = max(n_script_steps, args.cpu_steps + 8)      # the oracle leg replays the same scripts from step 0
-    cfg = base.scaled(steps=n_script_steps)
-    stream_cfg = cfg.scaled(seed=cfg.seed + 7919 * rank) if rank > 0 else cfg
+    cfg, stream_cfg = plan_rank(args, rank)
 
     t0 = time.time()
     corpus, logits, rowmax = make_inputs_gpu(cfg, device)
@@ -369,6 +484,7 @@ def run_ours(args):
         assert be.status() == 0
 
     all_tokens, max_ms = reduce_over_ranks(tokens, total_ms, world, device)
+    rank_seeds = gather_over_ranks(stream_cfg.seed, world)      # one distinct script seed per rank
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -408,19 +524,12 @@ def run_ours(args):
                 "note": f"{split['steps']} further steps of the same loop after the timed region, accept + walk + draft "
                         "in a kernel of its own (library events around it)", **split}
     st = W.trace_stats(cfg, stats_trace)
-    out = {
-        "metric": METRIC, "value": all_tokens / (max_ms / 1e3), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic",
-        "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.vocab, "min_match": cfg.min_match,
-                   "corpus_tokens": cfg.n_corpus, "accept_p": cfg.accept_p,
-                   "logits_bytes_per_step": R * cfg.vocab * 2,
-                   "l2": "inputs larger than L2 (logits re-read from HBM every step)" if R * cfg.vocab * 2 > 252e6
-                   else "inputs smaller than 2x L2: bandwidth figures are not HBM figures",
-                   "timing": "CUDA events around each sam_step on the launching stream, summed over steps; "
-                             "sparse logits planting between steps excluded; a spin kernel ahead of the first "
-                             "event keeps the queue full so host launch latency is not timed"},
+    out = headline(cfg, world, args, all_tokens, max_ms)
+    out.update({
+        "timing": "CUDA events around each sam_step on the launching stream, summed over steps, maximum over ranks; "
+                  "sparse logits planting between steps excluded; a spin kernel ahead of the first "
+                  "event keeps the queue full so host launch latency is not timed",
+        "rank_seeds": rank_seeds,
         "steps_per_s": args.steps / (max_ms / 1e3),
         "stream_steps_per_s": world * cfg.B * args.steps / (max_ms / 1e3),
         "gpu_launches": launches,
@@ -446,7 +555,7 @@ def run_ours(args):
                     "sam_build_tokens_per_s": cfg.n_corpus / t_build,
                     "states": index.n_states, "edges": index.n_edges, "device_bytes": index.device_bytes},
         "wall_s_timed_loop_incl_harness": wall,
-    }
+    })
     if args.cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(cfg, corpus, scripts, logits, rowmax, args.cpu_steps)
     print(json.dumps(out))
@@ -455,14 +564,20 @@ def run_ours(args):
 
 
 # ----------------------------------------------------------------------------- oracle arm
-def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads, single_thread_steps=0):
+def oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads, single_thread_steps=0, backend=None):
     """Times the oracle's step (wall clock, planting excluded) on the same closed loop; optionally goes on for a
-    few steps on one thread.  Returns (tokens, seconds, build seconds[, single-thread tokens, seconds])."""
-    import oracle
-    from tests.oracle_backend import OracleBackend
+    few steps on one thread.  Returns (tokens, seconds, build seconds[, single-thread tokens, seconds]).
+    `backend`: an OracleBackend to reuse (its automaton is kept, its stream state starts afresh)."""
+    from oracle.backend import OracleBackend
     feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
     t0 = time.time()
-    be = OracleBackend(cfg, corpus, host_bits, threads)
+    if backend is None:
+        be = OracleBackend(cfg, corpus, host_bits, threads)
+    else:
+        be = backend
+        be.state[:] = 0
+        be.mlen[:] = 0
+        be.threads = threads
     t_build = time.time() - t0
     toks, n = feeder.prime_tokens()
     drafts, n_draft = be.prime(toks, n)
@@ -504,34 +619,54 @@ def cpu_baseline(cfg, corpus, scripts, logits_dev, rowmax, steps):
             "argmax_GBps": cfg.rows * cfg.vocab * 2 * steps / secs / 1e9}
 
 
+REFERENCE_MAX_STEPS = 400      # oracle steps per run over all rank shares (about 20 s at the default workload)
+
+
 def run_reference(args):
+    """The oracle, as it stands, on the host cores: the work of all --gpus rank shares, one after the other (the
+    host cores are one pool, so the shares' times add up).  Under a launcher rank 0 alone does this."""
     rank, _, world = dist_env()
+    if world > 1 and world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if rank != 0:
         return
     import oracle
-    base = W.CONFIGS[args.config]
-    steps = min(args.steps, 40)
-    warmup = min(args.warmup, 3)
-    cfg = base.scaled(steps=warmup + steps + 1)
+    from oracle.backend import OracleBackend
+    n_shares = args.gpus
+    per_share_cap = max(1, REFERENCE_MAX_STEPS // n_shares)
+    steps = min(args.steps, per_share_cap)
+    warmup = min(args.warmup, per_share_cap)
+    cfg, _ = plan_rank(args, 0)
     corpus = W.make_corpus(cfg)
-    scripts = W.make_scripts(cfg, corpus)
     host_bits = W.make_noise_logits(cfg)
     rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(host_bits).max(axis=1))
     threads = oracle.host_threads()
-    tokens, secs, t_build = oracle_loop(cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads)
+    t0 = time.time()
+    be = OracleBackend(cfg, corpus, host_bits, threads)
+    t_build = time.time() - t0
+    tokens, secs, seeds = 0, 0.0, []
+    for r in range(n_shares):
+        _, stream_cfg = plan_rank(args, r)
+        scripts = W.make_scripts(stream_cfg, corpus)
+        tk, sc, _ = oracle_loop(stream_cfg, corpus, scripts, host_bits, rowmax, warmup, steps, threads, backend=be)
+        tokens += tk
+        secs += sc
+        seeds.append(stream_cfg.seed)
     v = tokens / secs
-    sample = (f"all {cfg.B} streams of {cfg.name}, {steps} closed-loop steps per run after {warmup} warm-up "
-              f"(requested {args.steps}/{args.warmup}; capped so the run stays within minutes)")
-    print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": warmup, "ms_per_step": secs / steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic",
-        "config": {"workload": cfg.name, "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.vocab, "min_match": cfg.min_match,
-                   "corpus_tokens": cfg.n_corpus},
-        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
-        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0, "oracle_build_s": t_build,
-    }))
+    capped = steps != args.steps or warmup != args.warmup
+    sample = (f"all {cfg.B} streams of each of {n_shares} rank share(s) of {cfg.name}, {steps} closed-loop steps per share "
+              f"after {warmup} warm-up" + (f" (requested {args.steps}/{args.warmup}; capped so the run stays within minutes)"
+                                          if capped else ""))
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": n_shares, "steps": steps,
+            "warmup": warmup, "ms_per_step": secs / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 compare / int32", "data": "synthetic", "config": workload_block(cfg),
+            "timing": "wall clock around each oracle step on the host cores, summed over steps and rank shares; "
+                      "planting between steps excluded",
+            "rank_seeds": seeds,
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "oracle_build_s": t_build}
+    print(json.dumps(line))
 
 
 # ----------------------------------------------------------------------------- growing index
@@ -543,7 +678,7 @@ def run_growing(args):
     import torch
     import paper_2512_18337_b200 as S
     from paper_2512_18337_b200.build import build
-    from tests.cuda_backend import CudaBackend
+    from harness.cuda_backend import CudaBackend
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -644,11 +779,9 @@ def run_vocab_parallel(args):
     import paper_2512_18337_b200 as S
     from paper_2512_18337_b200.build import build
     from paper_2512_18337_b200.parallel import reduce_argmax_keys, shard_bounds
-    from tests.cuda_backend import CudaBackend
+    from harness.cuda_backend import CudaBackend
 
-    rank, local_rank, world = dist_env()
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    rank, local_rank, world = init_ranks("nccl", args, lambda lr: torch.device(f"cuda:{lr}"))
     device = f"cuda:{local_rank}"
     torch.cuda.set_device(device)
     if rank == 0:
@@ -798,7 +931,7 @@ def run_multi(args):
     }))
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
@@ -806,7 +939,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index 0..5 (default 2: B=256, K=16; 5: the paper's evaluation shape, B=4, K=3)")
     ap.add_argument("--streams", type=int, default=0, help="override the workload's number of streams B (per GPU)")
-    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--e2e-steps", type=int, default=11,
+                    help="steps of each end-to-end loop through the host-buffer entry point (the first one warms "
+                         "the pinned path and is not timed)")
     ap.add_argument("--presleep-cycles", type=int, default=300000,
                     help="length of the spin kernel enqueued before each timed step (outside the events)")
     ap.add_argument("--variant", type=int, default=0, choices=[0, 1, 2, 3],
@@ -830,8 +965,20 @@ def main():
                     help="capture one sam_step in a CUDA graph after the warm-up and replay it for every timed step")
     ap.add_argument("--growing", action="store_true",
                     help="run the closed loop on a growing index instead (prints a separate JSON line)")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    return args
+
+
+def main():
+    args = parse_args()
+    from harness.launcher import spawn_ranks, under_launcher
+    single_process_modes = args.growing or args.multi > 0 or (args.impl == "reference")
+    if args.gpus > 1 and not under_launcher() and not single_process_modes:
+        # one process per GPU: this script again, under the torch launcher, with the same arguments
+        sys.exit(spawn_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
     elif args.growing:

@@ -63,10 +63,13 @@ typedef struct sam_index sam_index; /* opaque; owns the host-side automaton; dev
  * split happens; a clone copies transitions, suffix link and first end position.
  * Separators are ordinary symbols for construction and for the walk; they only stop draft
  * emission and are never emitted.
- *   corpus      host, n int32 tokens, 1 <= n <= 2^29
+ *   corpus      host, n int32 tokens, 1 <= n <= 2^29, every id in [0, 2^24) (the dense root table and the
+ *               hashed rows of the device layout are sized for 24-bit ids; other ids are refused here,
+ *               while the hot path itself takes any int32 and treats unknown ids as having no transition)
  *   separators  host, n_sep ids (0 <= n_sep <= SAM_MAX_SEPARATORS); may be NULL when n_sep = 0
  *   out         receives the handle; release it with sam_free
- * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOMEM. */
+ * Errors: SAM_ERR_INVALID_ARG (also: a token id outside [0, 2^24)), SAM_ERR_NOMEM, SAM_ERR_TOO_LARGE (the
+ * transitions of states with three or more successors do not fit 2^31 - 1 edge slots). */
 int sam_build(const int32_t* corpus, int64_t n, const int32_t* separators, int32_t n_sep,
               sam_index** out);
 
@@ -248,12 +251,18 @@ int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_con
  *   - All calls on a device share the one array, which keeps whatever the previous call left
  *     in it: two calls that overlap on the GPU (different streams, no ordering between them)
  *     race on it and return garbage.  Order them, or use sam_verify with separate workspaces.
+ *   - The array also holds the status word of the verification kernels (see sam_workspace_status);
+ *     every call clears it together with its rows, and sam_static_status reads it: 0 = the last
+ *     call on this device completed normally, otherwise a kernel gave up on a bounded wait and that
+ *     call's outputs are not valid (simply call again).  sam_static_status copies one int to the
+ *     host and synchronises the stream - a diagnostic that allocates nothing either.
  * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_TOO_LARGE, SAM_ERR_CUDA. */
 #define SAM_STATIC_MAX_ROWS   16384
 int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
                       const int32_t* drafts, const int32_t* n_draft,
                       int32_t* argmax_out, int32_t* accepted, int32_t* n_accepted,
                       void* cuda_stream);
+int sam_static_status(int32_t* status_out, void* cuda_stream);
 
 /* Host-buffer form of sam_step, for callers whose logits and bookkeeping live in host memory
  * (Algorithm 3, one loop iteration, end to end).  Copies logits [B*(K+1) rows, row_stride_elems
@@ -332,6 +341,13 @@ int sam_sync(sam_index* idx, void* cuda_stream, int64_t* tokens_on_device);
 /* What sam_sync has applied to the device so far: updates that scattered only what changed, updates
  * that copied a whole new image, and the host-to-device bytes of both.  Any pointer may be NULL. */
 int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_images, int64_t* bytes_copied);
+
+/* Forces the rare path of sam_sync: with every > 0, each every-th update the builder thread packs lays the
+ * wide rows out afresh and reaches the device as a whole image - what otherwise happens only when the
+ * wide-edge area fills up.  0 (the default) never forces it.  For tests and for measuring that path; takes
+ * effect with the next update the builder thread packs.  No counterpart in the paper.
+ * Errors: SAM_ERR_INVALID_ARG (not a growing index, every < 0). */
+int sam_growing_set_relayout_every(sam_index* idx, int64_t every);
 
 /* When the text grows, a state can be split, and a stream's (state, matched_len) may then name the
  * half that no longer holds its string.  This moves every state[b] (device, [B], in place) up its

@@ -1,4 +1,7 @@
-"""Closed-loop backend that runs every step with the CPU oracle (host logits)."""
+"""Closed-loop backend that runs every step with the CPU oracle (host logits).
+
+Test infrastructure like the rest of this package: used by the tests, the smoke check and the
+benchmark's CPU legs; it sequences oracle calls and holds the per-stream state, nothing more."""
 from __future__ import annotations
 
 import numpy as np

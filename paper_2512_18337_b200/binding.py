@@ -12,11 +12,8 @@ from typing import Optional
 
 import numpy as np
 
-import os
-
 _PKG = Path(__file__).resolve().parent
-# SAM_B200_LIB lets a tuning run point at another build of this same library
-_LIB_PATH = Path(os.environ.get("SAM_B200_LIB", _PKG / "libsam_b200.so"))
+_LIB_PATH = _PKG / "libsam_b200.so"
 _lib = None
 
 SAM_K_MAX = 32
@@ -53,6 +50,7 @@ _SIGNATURES = {
     "sam_argmax_partial": (C.c_int, [_vp, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sam_step_from_keys": (C.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "sam_verify_static": (C.c_int, [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "sam_static_status": (C.c_int, [C.POINTER(_i32), _vp]),
     "sam_step_host_staging_bytes": (_i64, [_i64, _i32, _i32, _i32]),
     "sam_step_host": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp, _i32, _vp, _vp, _vp, _i64, _vp]),
@@ -72,6 +70,7 @@ _SIGNATURES = {
     "sam_pending": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
     "sam_sync": (C.c_int, [_vp, _vp, C.POINTER(_i64)]),
     "sam_renormalize": (C.c_int, [_vp, _i32, _vp, _vp, _vp]),
+    "sam_growing_set_relayout_every": (C.c_int, [_vp, _i64]),
     "sam_update_stats": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
 }
 
@@ -87,6 +86,15 @@ class SamError(RuntimeError):
 
 def library_path() -> Path:
     return _LIB_PATH
+
+
+def use_library(path) -> None:
+    """Points the binding at another build of this same library (a tuning run comparing two builds, a test
+    of the missing-library error).  Only before the first call has loaded the default one."""
+    global _LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the library is already loaded")
+    _LIB_PATH = Path(path)
 
 
 def exported_symbols():
@@ -195,6 +203,11 @@ def sam_update_stats(handle: int):
     return a.value, b.value, c.value
 
 
+def sam_growing_set_relayout_every(handle: int, every: int) -> None:
+    """Every `every`-th update of a growing index is sent as a whole image (0: only when it has to be)."""
+    _check(_load().sam_growing_set_relayout_every(handle, every), "sam_growing_set_relayout_every")
+
+
 def sam_renormalize(handle: int, B: int, state, matched_len, stream=None) -> None:
     _check(_load().sam_renormalize(handle, B, _dev(state), _dev(matched_len), _stream(stream)), "sam_renormalize")
 
@@ -259,6 +272,13 @@ def sam_verify_static(logits, row_stride, B, K, V, drafts, n_draft, argmax_out, 
     _check(_load().sam_verify_static(_dev(logits), row_stride, B, K, V, _dev(drafts), _dev(n_draft),
                                      _dev(argmax_out), _dev(accepted), _dev(n_accepted), _stream(stream)),
            "sam_verify_static")
+
+
+def sam_static_status(stream=None) -> int:
+    """Status word of the last sam_verify_static call on the current device (0 = completed normally)."""
+    out = _i32(0)
+    _check(_load().sam_static_status(C.byref(out), _stream(stream)), "sam_static_status")
+    return int(out.value)
 
 
 def sam_step(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, accepted, n_accepted,

@@ -903,8 +903,9 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
                            n_accepted, keys, INT64_MAX);   // the array is sized for SAM_STATIC_MAX_ROWS rows
     if (rc != SAM_OK || B == 0) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    // whatever an earlier (possibly failed) call left behind, these rows start from zero
+    // whatever an earlier (possibly failed) call left behind, these rows and the status word start from zero
     SAM_CUDA(cudaMemsetAsync(keys, 0, static_cast<size_t>(rows) * 8, st));
+    SAM_CUDA(cudaMemsetAsync(keys + SAM_STATIC_MAX_ROWS, 0, sizeof(int), st));
     rc = launch_argmax(logits_bf16, row_stride_elems, rows, V, keys,
                        reinterpret_cast<int*>(keys + SAM_STATIC_MAX_ROWS), st);
     if (rc != SAM_OK) return rc;
@@ -915,6 +916,17 @@ int sam_verify_static(const void* logits_bf16, int64_t row_stride_elems, int32_t
     if (rc != SAM_OK) return rc;
     prof_mark(2, st);
     prof_done();
+    return SAM_OK;
+}
+
+int sam_static_status(int32_t* status_out, void* cuda_stream) {
+    if (!status_out) return SAM_ERR_INVALID_ARG;
+    unsigned long long* keys = nullptr;
+    const int rc = static_scratch(&keys);
+    if (rc != SAM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SAM_CUDA(cudaMemcpyAsync(status_out, keys + SAM_STATIC_MAX_ROWS, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SAM_CUDA(cudaStreamSynchronize(st));
     return SAM_OK;
 }
 
@@ -1057,6 +1069,11 @@ int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_i
     if (full_images) *full_images = idx->updates_full;
     if (bytes_copied) *bytes_copied = idx->update_bytes;
     return SAM_OK;
+}
+
+int sam_growing_set_relayout_every(sam_index* idx, int64_t every) {
+    if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
+    return dyn_set_relayout_every(idx, every);
 }
 
 int sam_renormalize(const sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream) {

@@ -17,6 +17,7 @@
 #include <deque>
 #include <mutex>
 #include <new>
+#include <atomic>
 #include <thread>
 #include <unordered_map>
 
@@ -34,7 +35,8 @@ struct DynIndex {
     std::vector<int32_t> packed_deg;           // per state: transitions its wide row held when it was last packed
     std::vector<Edge> mirror;                  // host copy of the device's wide array (rows sorted by token)
     int64_t w_used = 0;
-    int64_t compact_every = 0, updates_packed = 0;   // test knob: lay the wide rows out afresh at every k-th update
+    std::atomic<int64_t> relayout_every{0};    // > 0: lay the wide rows out afresh at every k-th update (sam_growing_set_relayout_every)
+    int64_t updates_packed = 0;
 
     std::thread worker;
     std::mutex mu;
@@ -234,7 +236,8 @@ int pack_changes(DynIndex& D, int64_t corpus_before, Delta* out) {
     out->rec_ids.reserve(b.dirty.size());
     out->recs.reserve(b.dirty.size());
     std::sort(b.redirected.begin(), b.redirected.end());
-    if (D.compact_every > 0 && ++D.updates_packed % D.compact_every == 0) {
+    const int64_t every = D.relayout_every.load();
+    if (every > 0 && ++D.updates_packed % every == 0) {
         Delta fresh;
         const int rc = pack_full(D, &fresh);
         *out = std::move(fresh);
@@ -324,14 +327,7 @@ int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tok
         // sorted rows sit in power-of-two slots (less than twice their length), hash rows are between an eighth
         // and a half full; 8 edges of room per token leaves ample slack for the corpora this is meant for, and
         // when the area does fill up the rows are laid out afresh (SAM_ERR_TOO_LARGE if even that does not fit)
-        if (const char* e = std::getenv("SAM_B200_COMPACT_EVERY")) D->compact_every = std::atoll(e);   // test knob
-        double per_token = 8.0;
-        if (const char* e = std::getenv("SAM_B200_WIDE_EDGES_PER_TOKEN")) {   // tuning / test knob
-            const double v = std::atof(e);
-            if (v >= 0.25 && v <= 64.0) per_token = v;
-        }
-        D->w_cap = std::min<int64_t>(static_cast<int64_t>(per_token * static_cast<double>(max_tokens)) + 1024,
-                                     (int64_t(1) << 31) - 64);
+        D->w_cap = std::min<int64_t>(8 * max_tokens + 1024, (int64_t(1) << 31) - 64);
         D->span_cap = static_cast<int64_t>(max_token_id) + 1;
         Builder& b = D->b;
         b.hash_alloc(1u << 16);
@@ -470,6 +466,13 @@ int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges) {
     D->cv_idle.wait(lk, [&] { return D->inbox.empty() && !D->busy; });
     if (n_states) *n_states = static_cast<int64_t>(D->b.len.size());
     if (n_edges) *n_edges = static_cast<int64_t>(D->b.e_tok.size());
+    return SAM_OK;
+}
+
+int dyn_set_relayout_every(sam_index* idx, int64_t every) {
+    DynIndex* D = idx->dyn;
+    if (!D || every < 0) return SAM_ERR_INVALID_ARG;
+    D->relayout_every.store(every);
     return SAM_OK;
 }
 

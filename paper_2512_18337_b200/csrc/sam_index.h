@@ -131,4 +131,5 @@ int dyn_full_image(sam_index* idx, Delta* out);                        // waits,
 int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges);    // waits; states / transitions right now
 int dyn_refresh_csr(sam_index* idx);                                   // waits, refills the flat arrays for sam_export
 void dyn_counts(sam_index* idx, int64_t* queued, int64_t* built);      // tokens handed in / tokens indexed on the host
+int dyn_set_relayout_every(sam_index* idx, int64_t every);             // every k-th update becomes a whole image (0: never forced)
 }  // namespace samb200

@@ -12,8 +12,8 @@ import torch
 
 import oracle
 import workload as W
-from tests.cuda_backend import CudaBackend
-from tests.oracle_backend import OracleBackend
+from harness.cuda_backend import CudaBackend
+from oracle.backend import OracleBackend
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"

@@ -13,8 +13,8 @@ import torch
 import oracle
 import paper_2512_18337_b200 as S
 import workload as W
-from tests.cuda_backend import CudaBackend, bits_to_device
-from tests.oracle_backend import OracleBackend
+from harness.cuda_backend import CudaBackend, bits_to_device
+from oracle.backend import OracleBackend
 
 pytestmark = pytest.mark.gpu
 

@@ -13,8 +13,8 @@ import torch
 import oracle
 import paper_2512_18337_b200 as S
 import workload as W
-from tests.cuda_backend import CudaBackend, bits_to_device
-from tests.oracle_backend import OracleBackend
+from harness.cuda_backend import CudaBackend, bits_to_device
+from oracle.backend import OracleBackend
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -42,16 +42,16 @@ def _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm):
     return d_o, nd_o
 
 
-@pytest.mark.parametrize("seed,compact_every", [(0, None), (1, "4")])
-def test_draft_parity_while_the_text_grows(seed, compact_every, monkeypatch):
-    """With the library's test knob set, every fourth update lays the wide rows out afresh and is sent as a whole
-    image (what happens by itself when the wide area fills up); the default keeps every update incremental."""
+@pytest.mark.parametrize("seed,compact_every", [(0, None), (1, 4)])
+def test_draft_parity_while_the_text_grows(seed, compact_every):
+    """With sam_growing_set_relayout_every(4), every fourth update lays the wide rows out afresh and is sent as a
+    whole image (what happens by itself when the wide area fills up); the default keeps every update incremental."""
     rng = np.random.default_rng(seed)
     sep, K, mm, B, ld = 1000, 6, 2, 48, 12
     text = _hub_text(rng, 3000, sep)
-    if compact_every is not None:
-        monkeypatch.setenv("SAM_B200_COMPACT_EVERY", compact_every)
     index = S.SamIndex(text, [sep], max_tokens=12000, max_token_id=sep + 50)
+    if compact_every is not None:
+        S.sam_growing_set_relayout_every(index.handle, compact_every)
     osam = oracle.OracleSAM(text, [sep])
     st = torch.zeros(B, dtype=torch.int32, device=DEV)
     ml = torch.zeros(B, dtype=torch.int32, device=DEV)

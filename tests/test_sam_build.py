@@ -198,9 +198,9 @@ def test_missing_library_fails_loudly(tmp_path):
     code = (
         "import os, sys\n"
         f"sys.path.insert(0, {ROOT!r})\n"
-        f"os.environ['SAM_B200_LIB'] = {str(tmp_path / 'nowhere.so')!r}\n"
         "import numpy as np\n"
         "import paper_2512_18337_b200 as S\n"
+        f"S.use_library({str(tmp_path / 'nowhere.so')!r})\n"
         "try:\n"
         "    S.sam_build(np.array([1, 2, 3], np.int32), [9])\n"
         "except RuntimeError as e:\n"

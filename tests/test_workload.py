@@ -5,7 +5,7 @@ import numpy as np
 
 import workload as W
 from tests import naive
-from tests.oracle_backend import OracleBackend
+from oracle.backend import OracleBackend
 
 
 def test_bf16_rounding():
