@@ -2,8 +2,10 @@
 
 TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's CPU
 baseline may import this; the CUDA product path never does, and this module
-imports nothing from the CUDA package.  All arithmetic lives in the C file;
-this wrapper only compiles it with gcc and marshals numpy arrays.
+imports nothing from the CUDA package.  The arithmetic of the single-automaton
+path lives in the C file, which this wrapper compiles with gcc and calls through
+numpy arrays; only the composite-drafting rule (`multi_draft`) is stated here in
+Python, on top of the C walk and draft.
 """
 from __future__ import annotations
 
@@ -82,6 +84,8 @@ def _load():
                                        _i32p, _i32p, C.c_uint32, _i64p]
         lib.oracle_speculation_enabled.restype = C.c_int32
         lib.oracle_speculation_enabled.argtypes = [C.c_int64] * 4
+        lib.oracle_speculation_pays.restype = C.c_int32
+        lib.oracle_speculation_pays.argtypes = [_i64p, C.c_int32, C.c_double]
         _lib = lib
     return _lib
 
@@ -195,6 +199,14 @@ SKIP_UNUSED_ROWS = 2
 
 def speculation_enabled(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:
     return bool(_load().oracle_speculation_enabled(context_len, batch_size, max_context_len, max_batch_size))
+
+
+def speculation_pays(counters: np.ndarray, K: int, cost_ratio: float) -> bool:
+    """The counter-driven switch: does the window of passes behind `counters` (int64[6] as oracle_step_ex fills
+    them) commit more tokens than it costs, a (K+1)-row pass costing cost_ratio one-row passes?"""
+    c = np.ascontiguousarray(counters, dtype=np.int64)
+    assert c.shape == (6,)
+    return bool(_load().oracle_speculation_pays(c.ctypes.data_as(_i64p), K, float(cost_ratio)))
 
 
 def argmax_row(row_bits: np.ndarray) -> int:

@@ -421,3 +421,21 @@ int32_t oracle_speculation_enabled(int64_t context_len, int64_t batch_size,
 {
     return !(context_len > max_context_len || batch_size > max_batch_size);
 }
+
+/* The switch driven by the running statistics (Section 5.4.3: speculation is switched off "when its overhead
+ * outweighs the gains"; Algorithm 3 step 4; Section 6.5 for OTE).  The paper leaves the rule to the deployment
+ * ("empirically determined" thresholds).  Reading taken here: a verification pass over one row costs 1, a pass
+ * over all K+1 rows costs cost_ratio (supplied by the caller from measurements), a pass over r rows lies on the
+ * line between the two, 1 + (cost_ratio - 1)(r - 1)/K; plain decoding commits one token per unit of cost.
+ * Speculation pays when the window of passes described by the counters committed more tokens than it cost:
+ *      sum(committed) > sum over passes of [1 + (cost_ratio - 1)(rows - 1)/K]
+ * With the counters of oracle_step_ex (committed - passes = accepted draft tokens) this is
+ *      accepted * K > (cost_ratio - 1) * (rows - passes),
+ * evaluated in double precision; when every pass reads all K+1 rows it is OTE > cost_ratio.
+ * A window without passes says nothing: speculation stays on. */
+int32_t oracle_speculation_pays(const int64_t *counters, int32_t K, double cost_ratio)
+{
+    const int64_t passes = counters[0], accepted = counters[3], rows = counters[5];
+    if (passes <= 0) return 1;
+    return (double)accepted * (double)K > (cost_ratio - 1.0) * (double)(rows - passes);
+}

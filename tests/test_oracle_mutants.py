@@ -69,6 +69,18 @@ MUTANTS = [
      "            next_n_draft[b] = 0;\n        } else {",
      "        if (0) {\n            for (int32_t j = 0; j < K; j++) nx[j] = -1;\n"
      "            next_n_draft[b] = 0;\n        } else {"),
+    ("the counter-driven switch speculates on a tie between tokens and cost",
+     "return (double)accepted * (double)K > (cost_ratio - 1.0) * (double)(rows - passes);",
+     "return (double)accepted * (double)K >= (cost_ratio - 1.0) * (double)(rows - passes);"),
+    ("the counter-driven switch charges the first row of a pass as an extra row",
+     "return (double)accepted * (double)K > (cost_ratio - 1.0) * (double)(rows - passes);",
+     "return (double)accepted * (double)K > (cost_ratio - 1.0) * (double)(rows);"),
+    ("the counter-driven switch forgets that the extra cost is spread over K rows",
+     "return (double)accepted * (double)K > (cost_ratio - 1.0) * (double)(rows - passes);",
+     "return (double)accepted > (cost_ratio - 1.0) * (double)(rows - passes);"),
+    ("the counter-driven switch compares all committed tokens with the extra cost",
+     "const int64_t passes = counters[0], accepted = counters[3], rows = counters[5];",
+     "const int64_t passes = counters[0], accepted = counters[1], rows = counters[5];"),
 ]
 
 _CHILD = r"""
