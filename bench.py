@@ -299,6 +299,7 @@ def run_ours(args):
     be.counters = torch.zeros(S.SAM_N_COUNTERS, dtype=torch.int64, device=device)
     if args.skip_unused_rows:
         be.flags |= S.SAM_STEP_SKIP_UNUSED_ROWS
+        be.chain_row_lists = True       # every step's accept kernel lists the rows of the next step: two launches per step
     toks, n = feeder.prime_tokens()
     drafts, n_draft = be.prime(toks, n)
 
@@ -727,8 +728,7 @@ def run_growing(args):
         if i >= 0:
             torch.cuda._sleep(args.presleep_cycles)
             ev[i][0].record()
-        S.sam_sync(index.handle)
-        S.sam_renormalize(index.handle, cfg.B, be.state, be.mlen)
+        S.sam_sync_renormalize(index.handle, cfg.B, be.state, be.mlen)
         be.launch_step()
         if i >= 0:
             ev[i][1].record()
@@ -755,7 +755,7 @@ def run_growing(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "dtype": "bf16 compare / int32", "data": "synthetic",
         "config": {"workload": cfg.name + " + one appended session per step (all committed tokens)",
-                   "B": cfg.B, "K": cfg.K, "V": cfg.vocab, "timing": "CUDA events around sam_sync + sam_renormalize + sam_step"},
+                   "B": cfg.B, "K": cfg.K, "V": cfg.vocab, "timing": "CUDA events around sam_sync_renormalize + sam_step"},
         "appended_tokens_per_step": appended / args.steps,
         "mean_tokens_not_yet_on_device_at_step_end": statistics.mean(lag),
         "updates": {"incremental": stats1[0] - stats0[0], "full_images": stats1[1] - stats0[1],
@@ -790,7 +790,7 @@ def run_vocab_parallel(args):
         dist.barrier()
     shards = world if world > 1 else args.vocab_shards
     mine = [rank] if world > 1 else list(range(shards))
-    cfg = W.CONFIGS[args.config].scaled(steps=args.warmup + args.steps + 1)
+    cfg, _ = plan_rank(args, 0)          # every rank holds a column shard of the SAME streams' logits
     corpus, logits, rowmax = make_inputs_gpu(cfg, device)       # same seed on every rank: same logits
     scripts = W.make_scripts(cfg, corpus)
     feeder = W.ClosedLoopFeeder(cfg, scripts, rowmax)
@@ -801,6 +801,7 @@ def run_vocab_parallel(args):
     keys = [torch.zeros(R + 1, dtype=torch.int64, device=device) for _ in mine]
     merged = torch.zeros(R, dtype=torch.int64, device=device)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    shard_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(mine) + 1)] for _ in range(args.steps)]
     tokens = 0
     for t in range(args.warmup + args.steps):
         ow = feeder.overwrites(t, drafts, n_draft)
@@ -809,9 +810,13 @@ def run_vocab_parallel(args):
         if i >= 0:
             torch.cuda._sleep(args.presleep_cycles)
             ev[i][0].record()
-        for k, r in zip(keys, mine):
+        for q, (k, r) in enumerate(zip(keys, mine)):
             lo, hi = shard_bounds(c.vocab, r, shards)
+            if i >= 0:
+                shard_ev[i][q].record()
             S.sam_argmax_partial(be.logits.data_ptr() + 2 * lo, be.stride, R, hi - lo, lo, k)
+        if i >= 0:
+            shard_ev[i][len(mine)].record()
         if world > 1:
             reduce_argmax_keys(keys[0], R)
             words = keys[0]
@@ -833,9 +838,17 @@ def run_vocab_parallel(args):
             tokens += int(n_acc.sum())
     ms = float(sum(a.elapsed_time(b) for a, b in ev))
     _, ms = reduce_over_ranks(0, ms, world, device)
+    # one shard's sam_argmax_partial (zero-fill of its words + the argmax kernel), from the events between the calls
+    shard_ms = [e[q].elapsed_time(e[q + 1]) for e in shard_ev for q in range(len(mine))]
+    shard_bytes = [R * (2 * (shard_bounds(c.vocab, r, shards)[1] - shard_bounds(c.vocab, r, shards)[0]) + 4) for r in mine]
+    peak, peak_kind = measured_peaks()
     if rank == 0:
+        per_shard_gbs = statistics.mean(shard_bytes) / (statistics.mean(shard_ms) * 1e-3) / 1e9
         print(json.dumps({
-            "metric": METRIC + "_vocab_parallel", "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC + "_vocab_parallel",
+            "shard_argmax": {"us_per_shard": statistics.mean(shard_ms) * 1e3, "GBps": per_shard_gbs, "frac": per_shard_gbs / peak,
+                             "peak_kind": f"of {peak_kind}", "bytes_per_shard": statistics.mean(shard_bytes),
+                             "note": "events around each sam_argmax_partial call (memset of the words + argmax kernel)"}, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "strong", "dtype": "bf16 compare / int32", "data": "synthetic",
             "config": {"workload": cfg.name, "B": c.B, "K": c.K, "V": c.vocab, "vocab_shards": shards,

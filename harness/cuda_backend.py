@@ -31,6 +31,8 @@ class CudaBackend:
         self.accepted = torch.full((B, K + 1), -7, **i32)
         self.n_accepted = torch.zeros(B, **i32)
         self.flags = 0              # SAM_STEP_* options used by launch_step
+        self.chain_row_lists = False  # with SAM_STEP_SKIP_UNUSED_ROWS: let each step list the rows of the next one
+        self._list_ready = False
         self.counters = None        # optional int64[SAM_N_COUNTERS] device tensor
         self.ws_bytes = S.sam_workspace_bytes(B, K)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
@@ -62,9 +64,15 @@ class CudaBackend:
     def launch_step(self):
         """Enqueue one fused step on the current stream (drafts/n_draft are updated in place)."""
         c = self.cfg
+        flags = self.flags
+        if self.chain_row_lists and (flags & S.SAM_STEP_SKIP_UNUSED_ROWS):
+            # drafts / n_draft are fed straight back, so from the second step on the previous step's list is the one
+            if self._list_ready:
+                flags |= S.SAM_STEP_ROW_LIST_READY
+            self._list_ready = True
         S.sam_step_ex(self.index.handle, self.logits, self.stride, c.B, c.K, c.vocab, self.drafts, self.n_draft,
                       self.argmax, self.accepted, self.n_accepted, self.state, self.mlen, c.min_match,
-                      self.drafts, self.n_draft, self.flags, self.counters, self.ws, self.ws_bytes)
+                      self.drafts, self.n_draft, flags, self.counters, self.ws, self.ws_bytes)
 
     def status(self) -> int:
         return S.sam_workspace_status(self.ws, self.cfg.B, self.cfg.K)

@@ -111,7 +111,7 @@ int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
 /* Reads the status word the verification kernels keep inside the scratch: 0 = fine,
  * 1 = a kernel gave up on one of its internal (bounded) waits, 2 = a kernel was handed more
  * finished streams than its internal queue holds (the host sizes the launch so that this does not
- * happen).  After a non-zero status the outputs of that call are not valid - re-initialise the
+ * happen), 3 = SAM_STEP_ROW_LIST_READY was given but the scratch holds no row list for this batch shape.  After a non-zero status the outputs of that call are not valid - re-initialise the
  * scratch and retry.  Copies one int to the host and synchronises the stream: a diagnostic, not a
  * hot-path call.  B and K locate the word (same values as in the calls that used the scratch). */
 int sam_workspace_status(const void* workspace, int32_t B, int32_t K, int32_t* status_out, void* cuda_stream);
@@ -179,6 +179,16 @@ int sam_step(const sam_index* idx,
  *       model's own token after a full accept); argmax_out of the rows beyond is -1.  A small kernel
  *       lists the used rows first, then the argmax kernel streams only those - the bytes read per call
  *       drop from B*(K+1) rows to sum(n_draft)+B rows.
+ *   SAM_STEP_ROW_LIST_READY   (sam_step_ex only, together with SAM_STEP_SKIP_UNUSED_ROWS) the caller states
+ *       that the previous call through this workspace was a sam_step_ex with SAM_STEP_SKIP_UNUSED_ROWS for
+ *       the same B and K, and that drafts / n_draft are what that call wrote to next_drafts / next_n_draft,
+ *       unmodified.  Every such call leaves the list of the rows its successor needs in the workspace (its
+ *       accept kernel writes it as a by-product), so the listing kernel is not launched: two launches per
+ *       step instead of three.  If the workspace holds no list for this B and K (first call, workspace
+ *       re-initialised, another shape in between) nothing is reduced, the outputs of the call are not
+ *       valid and the status word reads 3 (sam_workspace_status); a list that is stale in any other way
+ *       gives the results of the rows it names - wrong for this call, but every access stays inside the
+ *       caller's buffers.
  *   counters  device, int64[SAM_N_COUNTERS], 8-byte aligned, or NULL.  Every call ADDS, per stream:
  *       [0] verification passes (1), [1] committed tokens, [2] proposed draft tokens, [3] accepted draft
  *       tokens, [4] non-empty proposals, [5] logits rows read.  Section 6.5: OTE = [1]/[0],
@@ -187,6 +197,7 @@ int sam_step(const sam_index* idx,
  * Everything else is as in sam_verify / sam_step, which are these calls with flags = 0, counters = NULL. */
 #define SAM_STEP_NO_SPECULATION   1u
 #define SAM_STEP_SKIP_UNUSED_ROWS 2u
+#define SAM_STEP_ROW_LIST_READY   4u
 #define SAM_N_COUNTERS            6
 int sam_verify_ex(const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
                   const int32_t* drafts, const int32_t* n_draft,
@@ -231,6 +242,23 @@ int sam_step_from_keys(const sam_index* idx, int64_t* keys, int32_t B, int32_t K
  * thresholds are deployment-specific ("empirically determined" in the paper); a host-side helper,
  * no device work. */
 int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_context_len, int64_t max_batch_size);
+
+/* The same decision taken from the running statistics instead of fixed thresholds (Section 5.4.3: speculation is
+ * disabled "when its overhead outweighs the gains"; Section 6.5: OTE).  The paper leaves the rule to the
+ * deployment; the one here prices a verification pass over r of the K+1 rows at 1 + (cost_ratio - 1)(r - 1)/K
+ * one-row passes - cost_ratio, the measured cost of a full (K+1)-row pass relative to a one-row pass, comes from
+ * the caller - and keeps speculating when the passes behind the counters committed more tokens than they cost
+ * (plain decoding commits one token per one-row pass):
+ *     accepted draft tokens * K  >  (cost_ratio - 1) * (rows read - passes)      in double precision;
+ * with all K+1 rows read in every pass this is OTE > cost_ratio.
+ *   counters    HOST, int64[SAM_N_COUNTERS]: a copy of the device counters of sam_step_ex / sam_verify_ex over
+ *               the window to judge (the caller zeroes them, or subtracts two readings); only passes [0],
+ *               accepted draft tokens [3] and rows read [5] are used.  Take them from passes that did speculate:
+ *               passes with SAM_STEP_NO_SPECULATION show OTE = 1 by construction, so a caller that has switched
+ *               speculation off should try it again from time to time.
+ *   K           the draft length those passes used, 1..SAM_K_MAX;  cost_ratio > 0
+ * Returns 1 (speculate), 0 (do not), or SAM_ERR_INVALID_ARG.  A window without passes returns 1.  Host only. */
+int sam_speculation_pays(const int64_t* counters, int32_t K, double cost_ratio);
 
 /* Allocation-free form of sam_verify (a packaging variant; the paper has no counterpart).
  * Some callers cannot obtain device scratch at all: a plugin running inside a serving engine
@@ -282,9 +310,10 @@ int sam_step_host(const sam_index* idx,
                   int32_t* next_drafts, int32_t* next_n_draft,
                   void* staging, int64_t staging_bytes, void* cuda_stream);
 
-/* sam_step_host with step options (SAM_STEP_*).  With SAM_STEP_SKIP_UNUSED_ROWS only rows 0..n_draft[b]
- * of every stream are copied to the device (one copy per stream) - the host-to-device traffic, which
- * dominates this call, shrinks with the proposals. */
+/* sam_step_host with step options (SAM_STEP_*; SAM_STEP_ROW_LIST_READY is not accepted here).  With
+ * SAM_STEP_SKIP_UNUSED_ROWS only rows 0..n_draft[b] of every stream are copied to the device (one copy per
+ * run of rows that touch or nearly touch) - the host-to-device traffic, which dominates this call, shrinks
+ * with the proposals. */
 int sam_step_host_ex(const sam_index* idx,
                      const void* logits_bf16, int64_t row_stride_elems, int32_t B, int32_t K, int32_t V,
                      const int32_t* drafts, const int32_t* n_draft,
@@ -303,7 +332,7 @@ int sam_step_host_ex(const sam_index* idx,
  * sam_build_growing builds the automaton of corpus[0..n) (n may be 0) like sam_build, keeps the
  * builder alive in a thread of its own, and sizes the device blob (sam_sizes) for up to max_tokens
  * tokens: room for 2*max_tokens+2 state records, 8*max_tokens wide edges, a dense root table for token ids
- * 0..max_token_id, the text, and an 8 MiB staging area for updates.  sam_upload, sam_draft,
+ * 0..max_token_id, the text, an 8 MiB staging area for large updates and eight 1 MiB slots for small ones.  sam_upload, sam_draft,
  * sam_verify, sam_step, sam_export, sam_sizes and sam_free work as for any other index.
  *   max_tokens    1 .. 2^29, >= n;  max_token_id  largest token id that will ever be indexed
  *                 (separators included), < 2^24
@@ -325,18 +354,32 @@ int sam_extend(sam_index* idx, const int32_t* tokens, int64_t n);
 int sam_pending(sam_index* idx, int64_t* tokens_queued, int64_t* tokens_built, int64_t* tokens_on_device);
 
 /* Brings the device copy up to date with everything the builder thread has finished: the records
- * of changed states, rewritten wide rows, changed root entries and the appended text are copied
- * into the blob's staging area and scattered by small kernels on the stream (a whole new image is
- * copied instead after the wide-edge area had to be laid out afresh).  Does not wait for the
- * builder thread and does not synchronise the stream; hot-path calls enqueued afterwards on the
- * same stream see the grown automaton.  Call it from the thread that makes the hot-path calls.
- * The first small update creates 1 MiB of page-locked host memory and an event for the handle
- * (released by sam_free); a later call may wait on the host until the previous update's copy has
- * left that buffer.
- * After it, run sam_renormalize on every batch of stream states that will be used again.
+ * of changed states, rewritten wide rows, changed root entries and the appended text are scattered
+ * into the live arrays by a small kernel on the stream (a whole new image is copied instead after
+ * the wide-edge area had to be laid out afresh).  Does not wait for the builder thread and does not
+ * synchronise the stream; hot-path calls enqueued afterwards on the same stream see the grown
+ * automaton.  Call it from the thread that makes the hot-path calls.
+ * Where the bytes travel: an update of up to 1 MiB (what accumulates between two decoding steps) has
+ * normally been copied into one of the blob's slots already, by the builder thread, through page-locked
+ * memory on a stream the library owns (both created by sam_upload of a growing index, released by
+ * sam_free), while earlier steps were running; sam_sync then only makes the caller's stream wait for
+ * that copy's event and launches the scatter kernel.  The copy touches nothing a kernel reads; every
+ * write into live records, rows, root table and text happens in the scatter kernel, in stream order
+ * between the step before and the step after.  An update that was not sent ahead (no free slot, or
+ * larger than a slot) is copied on the caller's stream instead, as before.
+ * After it, run sam_renormalize on every batch of stream states that will be used again - or use
+ * sam_sync_renormalize, which does both.
  * Errors: SAM_ERR_INVALID_ARG, SAM_ERR_NOT_UPLOADED, SAM_ERR_TOO_LARGE (the automaton no longer
  * fits the blob), SAM_ERR_CUDA. */
 int sam_sync(sam_index* idx, void* cuda_stream, int64_t* tokens_on_device);
+
+/* sam_sync followed by sam_renormalize(idx, B, state, matched_len) in as few launches as possible: when
+ * the last pending update is a small one, the block of its scatter kernel that finishes last repairs the
+ * stream states, so ONE kernel stands between the previous decoding step and the next; when nothing is
+ * pending nothing is launched (states only need repair after growth).  Same results as the two calls.
+ * Errors: as sam_sync and sam_renormalize. */
+int sam_sync_renormalize(sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream,
+                         int64_t* tokens_on_device);
 
 /* What sam_sync has applied to the device so far: updates that scattered only what changed, updates
  * that copied a whole new image, and the host-to-device bytes of both.  Any pointer may be NULL. */

@@ -38,6 +38,7 @@ _SIGNATURES = {
     "sam_step_ex": (C.c_int, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                               _vp, _vp, _i32, _vp, _vp, C.c_uint32, _vp, _vp, _i64, _vp]),
     "sam_adaptive_switch": (C.c_int, [_i64, _i64, _i64, _i64]),
+    "sam_speculation_pays": (C.c_int, [_vp, _i32, C.c_double]),
     "sam_set_bytes": (_i64, [_i32]),
     "sam_set_create": (C.c_int, [_vp, _i32, _vp, _i64, _vp, C.POINTER(_vp)]),
     "sam_set_refresh": (C.c_int, [_vp, _vp]),
@@ -70,6 +71,7 @@ _SIGNATURES = {
     "sam_pending": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
     "sam_sync": (C.c_int, [_vp, _vp, C.POINTER(_i64)]),
     "sam_renormalize": (C.c_int, [_vp, _i32, _vp, _vp, _vp]),
+    "sam_sync_renormalize": (C.c_int, [_vp, _i32, _vp, _vp, _vp, C.POINTER(_i64)]),
     "sam_growing_set_relayout_every": (C.c_int, [_vp, _i64]),
     "sam_update_stats": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
 }
@@ -196,6 +198,15 @@ def sam_sync(handle: int, stream=None) -> int:
     return int(n.value)
 
 
+def sam_sync_renormalize(handle: int, B: int, state, matched_len, stream=None) -> int:
+    """sam_sync and sam_renormalize in one call (one kernel when the pending update is small); returns the
+    tokens visible on the device."""
+    n = _i64()
+    _check(_load().sam_sync_renormalize(handle, B, _dev(state), _dev(matched_len), _stream(stream), C.byref(n)),
+           "sam_sync_renormalize")
+    return int(n.value)
+
+
 def sam_update_stats(handle: int):
     """(incremental updates, whole-image updates, bytes copied) applied by sam_sync so far."""
     a, b, c = _i64(), _i64(), _i64()
@@ -291,6 +302,7 @@ def sam_step(handle, logits, row_stride, B, K, V, drafts, n_draft, argmax_out, a
 
 SAM_STEP_NO_SPECULATION = 1
 SAM_STEP_SKIP_UNUSED_ROWS = 2
+SAM_STEP_ROW_LIST_READY = 4
 SAM_N_COUNTERS = 6
 
 
@@ -385,6 +397,17 @@ def sam_multi_step(set_handle, logits, row_stride, B, K, V, drafts, n_draft, arg
 
 def sam_adaptive_switch(context_len: int, batch_size: int, max_context_len: int, max_batch_size: int) -> bool:
     return bool(_load().sam_adaptive_switch(context_len, batch_size, max_context_len, max_batch_size))
+
+
+def sam_speculation_pays(counters, K: int, cost_ratio: float) -> bool:
+    """Counter-driven switch; `counters` is a HOST int64[SAM_N_COUNTERS] array (a copy of the device counters)."""
+    c = np.ascontiguousarray(counters, dtype=np.int64)
+    if c.shape != (SAM_N_COUNTERS,):
+        raise ValueError("expected SAM_N_COUNTERS int64 values")
+    r = _load().sam_speculation_pays(c.ctypes.data, K, float(cost_ratio))
+    if r < 0:
+        raise SamError(int(r), "sam_speculation_pays")
+    return bool(r)
 
 
 def _hostptr(a) -> Optional[int]:

@@ -4,8 +4,17 @@
 // shared-memory stages with 1-D bulk asynchronous copies (cp.async.bulk, completion counted on
 // an mbarrier); the consumer warps reduce the tiles straight out of shared memory.  Loads cost
 // no issue slots and no registers, ~190 KB per SM are in flight, and the reduction of one tile
-// overlaps the copies of the following ones.  Requires 16-byte aligned rows (base and stride);
-// the direct-load kernel covers everything else.
+// overlaps the copies of the following ones.  Requires 16-byte aligned rows (base and stride) of at
+// least one 16-byte vector; the direct-load kernel covers everything else.
+//
+// How the consumer warps share the tiles depends on the tile size (BulkPlan, chosen by the host).  A tile
+// costs the consumers 0.58 us whatever its size - waking up on the barrier, the vote, locating the new
+// maximum, releasing the stage - beside 0.69 us per 64 KB (measured with eight warps on every tile).  With
+// tiles of about 60 KB (a 304 KB row cut in five) that keeps pace with HBM, and eight warps work on one tile
+// after the other.  With smaller tiles (the 76 KB row pieces of a vocabulary shard cut in two) it does not:
+// there the twelve consumer warps form three groups, tile k goes to group k mod 3, and the fixed cost of one
+// group's tile runs while the other groups are busy with theirs; the ring then has as many stages as fit
+// (five of 38 KB), so that the bytes in flight stay the same.
 //
 // The consumer warps never touch global memory for their results: when a row (or the CTA's part of
 // it) is finished, each warp leaves its candidate in a small ring in shared memory and moves on.
@@ -29,6 +38,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <type_traits>
 
 #include "sam_kernels.cuh"
 
@@ -40,25 +50,57 @@ namespace samb200 {
 #ifndef SAM_BULK_STAGES
 #define SAM_BULK_STAGES 3
 #endif
-#ifndef SAM_BULK_CONSUMER_WARPS
-#define SAM_BULK_CONSUMER_WARPS 8
-#endif
-constexpr int kBulkTileVec = SAM_BULK_TILE_VEC;        // capacity of one stage in 16-byte vectors (64 KB)
+constexpr int kBulkTileVec = SAM_BULK_TILE_VEC;        // largest tile in 16-byte vectors (64 KB)
 constexpr int kBulkTileBytes = kBulkTileVec * 16;
-constexpr int kBulkStages = SAM_BULK_STAGES;           // ring of kBulkStages * kBulkTileBytes (<= ~200 KB)
+constexpr int kBulkStages = SAM_BULK_STAGES;           // the ring holds kBulkStages * kBulkTileBytes (<= ~200 KB) ...
+constexpr int kBulkRingBytes = kBulkStages * kBulkTileBytes;
+constexpr int kMaxStages = 8;                          // ... cut into up to kMaxStages stages when the tiles are small
+#ifndef SAM_BULK_CONSUMER_WARPS
+#define SAM_BULK_CONSUMER_WARPS 12
+#endif
 constexpr int kBulkConsumerWarps = SAM_BULK_CONSUMER_WARPS;
 constexpr int kBulkConsumers = kBulkConsumerWarps * 32;
+constexpr int kWideGroupWarps = 8;                     // one group of eight warps on every tile (large tiles)
+constexpr int kSmallGroupWarps = 4;                    // groups of four warps taking tiles in turn (small tiles):
+constexpr int kSmallGroups = kBulkConsumerWarps / kSmallGroupWarps;   // three of them
+#ifndef SAM_BULK_SMALL_TILE_BYTES
+#define SAM_BULK_SMALL_TILE_BYTES (48 * 1024)
+#endif
+constexpr int kSmallTileBytes = SAM_BULK_SMALL_TILE_BYTES;   // below this a tile counts as small
+static_assert(kWideGroupWarps <= kBulkConsumerWarps && kSmallGroups * kSmallGroupWarps <= kBulkConsumerWarps, "consumer warps");
+
+// How the rows are tiled and how the consumer warps share the tiles (filled in by bulk_plan on the host).
+struct BulkPlan {
+    int tiles_per_row;     // a row is cut into this many tiles of tile_vec vectors (the last one may be shorter)
+    int tile_vec;
+    int n_stages;          // stages of stage_bytes bytes in the ring
+    int stage_bytes;
+    int n_groups;          // consumer groups; tile k of a CTA is reduced by group k mod n_groups
+    int group_warps;       // warps per group
+};
+inline BulkPlan bulk_plan(int V) {
+    BulkPlan p;
+    const long long nvec = V / 8;
+    p.tiles_per_row = static_cast<int>((nvec + kBulkTileVec - 1) / kBulkTileVec);
+    p.tile_vec = static_cast<int>((nvec + p.tiles_per_row - 1) / p.tiles_per_row);   // nearly equal tiles
+    p.stage_bytes = (p.tile_vec * 16 + 127) & ~127;
+    const bool small = p.stage_bytes < kSmallTileBytes;
+    p.n_groups = small ? kSmallGroups : 1;
+    p.group_warps = small ? kSmallGroupWarps : kWideGroupWarps;
+    p.n_stages = kBulkRingBytes / p.stage_bytes;
+    if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
+    return p;
+}
 constexpr int kBulkWalkerWarps = 2;                    // spare warps that walk ahead along the drafts
 constexpr int kBulkThreads = kBulkConsumers + 64 + kBulkWalkerWarps * 32;   // consumers, producer, finisher, walkers
 constexpr int kRowSlots = 64;                          // ring of per-row candidate slots (consumers -> finisher)
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kQueueCap = 1024;                        // streams one CTA can be handed (host checks the bound)
-constexpr size_t kBulkCtrlOff = static_cast<size_t>(kBulkStages) * kBulkTileBytes;
+constexpr size_t kBulkCtrlOff = static_cast<size_t>(kBulkRingBytes);
 constexpr size_t kBulkQueueOff = kBulkCtrlOff + 1024;
 constexpr size_t kBulkCandOff = kBulkQueueOff + kQueueCap * 4;
 constexpr size_t kBulkSmemBytes = kBulkCandOff + static_cast<size_t>(kRowSlots) * kBulkConsumerWarps * 8;
 
-enum : int { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusQueueOverflow = 2 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -112,8 +154,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
 }
 
 struct BulkShared {
-    uint64_t full[kBulkStages];
-    uint64_t empty[kBulkStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     long long issued;                 // tiles the producer has issued copies for
     int abort;
     int q_tail;                       // streams pushed into the queue
@@ -177,14 +219,14 @@ __device__ __forceinline__ void serve_queue(const DeviceSam& sam, const FusedTai
 
 __global__ void __launch_bounds__(kBulkThreads, 1)
 argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, long long R, int V,
-                   int tiles_per_row, int tile_vec, unsigned long long* __restrict__ keys,
+                   const __grid_constant__ BulkPlan plan, unsigned long long* __restrict__ keys,
                    int* __restrict__ status, const __grid_constant__ DeviceSam sam,
                    const __grid_constant__ PreWalk pw, const __grid_constant__ FusedTail ft,
                    const __grid_constant__ RowMap rm) {
-    // tile_vec <= kBulkTileVec: vectors per tile, chosen by the host so that a row splits into
-    // tiles_per_row nearly equal tiles (large tiles amortise the per-tile hand-shake best).
+    const int tiles_per_row = plan.tiles_per_row, tile_vec = plan.tile_vec, ns = plan.n_stages;
+    const int n_cons = plan.n_groups * plan.group_warps;                      // consumer warps that take part
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    unsigned char* stage_base = smem_raw;                                      // kBulkStages tiles
+    unsigned char* stage_base = smem_raw;                                      // ns stages of plan.stage_bytes
     BulkShared* sh = reinterpret_cast<BulkShared*>(smem_raw + kBulkCtrlOff);
     int* queue = reinterpret_cast<int*>(smem_raw + kBulkQueueOff);
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem_raw + kBulkCandOff);   // [kRowSlots][warps]
@@ -194,7 +236,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     // with a row list the number of rows is only known on the device, and a CTA's share may be empty
-    const long long n_all = (rm.list != nullptr) ? __ldg(rm.n_rows) : R;
+    const long long n_all = (rm.list != nullptr) ? listed_rows(rm, R) : R;
     const long long total = n_all * tiles_per_row;
     const long long t0 = total * blockIdx.x / gridDim.x;
     const long long t1 = total * (blockIdx.x + 1) / gridDim.x;
@@ -204,9 +246,9 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
     const int ragged = V & 7;                  // trailing elements read with plain loads
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kBulkStages; ++s) {
+        for (int s = 0; s < ns; ++s) {
             mbar_init(&sh->full[s], 1);
-            mbar_init(&sh->empty[s], kBulkConsumerWarps);
+            mbar_init(&sh->empty[s], plan.group_warps);
         }
         sh->abort = 0;
         sh->issued = 0;
@@ -222,6 +264,12 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         for (int i = threadIdx.x; i < kQueueCap; i += blockDim.x) queue[i] = -1;
     __syncthreads();
     volatile int* abort = &sh->abort;
+    // a row named by a list is clamped into the logits: a stale or foreign list can give wrong results, never a fault
+    auto actual_row = [&](long long pos) -> long long {
+        if (rm.list == nullptr) return pos;
+        const long long r = __ldg(rm.list + pos);
+        return r < 0 ? 0 : (r >= R ? R - 1 : r);
+    };
 
     if (warp == kBulkConsumerWarps) {
         // ------------------------------------------------------------------ producer
@@ -235,20 +283,20 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             const uint64_t policy = l2_evict_first_policy();
             for (long long t = t0; t < t1; ++t, ++it) {
                 // with a row list the row number is fetched before the wait, off the path of the copy
-                const long long arow = (rm.list != nullptr) ? __ldg(rm.list + row) : row;
+                const long long arow = actual_row(row);
                 if (!mbar_wait_bounded(&sh->empty[s], (use & 1u) ^ 1u, abort)) { ok = false; break; }
                 const int v0 = tile * tile_vec;
                 const int nv = max(0, min(tile_vec, nvec_row - v0));
                 if (nv > 0) {
                     const uint32_t bytes = static_cast<uint32_t>(nv) * 16u;
                     mbar_arrive_expect_tx(&sh->full[s], bytes);
-                    bulk_load(stage_base + static_cast<size_t>(s) * kBulkTileBytes,
+                    bulk_load(stage_base + static_cast<size_t>(s) * plan.stage_bytes,
                               reinterpret_cast<const uint4*>(logits + arow * stride) + v0, bytes, &sh->full[s], policy);
                 } else {
                     mbar_arrive(&sh->full[s]);      // nothing to copy (row shorter than one vector)
                 }
                 if (++tile == tiles_per_row) { tile = 0; ++row; }
-                if (++s == kBulkStages) { s = 0; ++use; }
+                if (++s == ns) { s = 0; ++use; }
             }
             sh->issued = it;
             if (!ok) {
@@ -262,7 +310,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         int done_rows = 0;
         uint32_t polls = 0;
         while (done_rows < n_rows) {
-            int p = (lane < kBulkConsumerWarps) ? ld_volatile_s32(&sh->prog[lane]) : 0x7fffffff;
+            int p = (lane < n_cons) ? ld_volatile_s32(&sh->prog[lane]) : 0x7fffffff;
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) p = min(p, __shfl_xor_sync(kFull, p, d));
             if (p <= done_rows) {                      // nothing new: every warp must have handed the row over
@@ -282,12 +330,12 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             const int n = min(32, p - done_rows);
             if (lane < n) {
                 const int i = done_rows + lane;
-                const long long row = (rm.list != nullptr) ? __ldg(rm.list + row_first + i) : row_first + i;
+                const long long row = actual_row(row_first + i);
                 const unsigned long long* c = cand + static_cast<size_t>(i % kRowSlots) * kBulkConsumerWarps;
                 unsigned long long k = 0ull;
 #pragma unroll
                 for (int w = 0; w < kBulkConsumerWarps; ++w) {
-                    const unsigned long long x = c[w];
+                    const unsigned long long x = (w < n_cons) ? c[w] : 0ull;
                     k = (x > k) ? x : k;
                 }
                 if (k != 0ull) atomicMax(keys + row, k);
@@ -351,22 +399,18 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         if (ft.mode != 0) serve_queue(sam, ft, sh, queue, abort, status, lane);
     } else {
         // ------------------------------------------------------------------ consumers
-        const int ct = threadIdx.x;                       // 0 .. kBulkConsumers-1
-        long long cur_row = -1;
+        bool ok = true;
         float best = __int_as_float(0xff800000);          // -inf: only strictly greater values are candidates
         int best_idx = -1;
-        bool first_nan = false;                           // element 0 of the current row is NaN (seen by thread 0 only)
-        bool ok = true;
-
-        // Hands the finished row over to the finisher: candidate into the row's slot, then the progress counter.
-        auto flush = [&]() -> bool {
-            if (cur_row < 0) return true;
+        bool first_nan = false;                           // element 0 of the current row is NaN (seen by one thread only)
+        // Hands this warp's candidate for the CTA's row number i over to the finisher: into the row's slot, then the
+        // progress counter.  Every taking-part consumer warp hands over every row of the CTA, in order.
+        auto hand_over = [&](int i) -> bool {
             unsigned long long k = (best_idx >= 0) ? pack_candidate(best, static_cast<unsigned>(best_idx + rm.v_offset)) : 0ull;
             if (first_nan) k = kCandidateFirstIsNaN;
             k = warp_max_u64(k);
             int good = 1;
             if (lane == 0) {
-                const int i = static_cast<int>(cur_row - row_first);
                 uint32_t polls = 0;
                 while (i - ld_volatile_s32(&sh->fin_rows) >= kRowSlots) {     // ring full: the finisher is behind
                     if (*abort || ++polls > kMaxPolls) { good = 0; break; }
@@ -378,33 +422,21 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                     st_volatile_s32(&sh->prog[warp], i + 1);
                 }
             }
+            best = __int_as_float(0xff800000);
+            best_idx = -1;
+            first_nan = false;
             return __shfl_sync(kFull, good, 0) != 0;
         };
-
-        long long row = row_first;
-        int tile = static_cast<int>(t0 - row * tiles_per_row);
-        int s = 0;
-        uint32_t use = 0;
-        for (long long t = t0; t < t1; ++t) {
-            if (row != cur_row) {
-                if (!flush()) { ok = false; break; }
-                cur_row = row;
-                best = __int_as_float(0xff800000);
-                best_idx = -1;
-                first_nan = false;
-            }
-            // the outcome of the wait is made uniform so that the warp leaves the loop together
-            if (!__all_sync(kFull, mbar_wait_bounded(&sh->full[s], use & 1u, abort))) { ok = false; break; }
-            const int v0 = tile * tile_vec;
-            const int nv = max(0, min(tile_vec, nvec_row - v0));
-            const uint4* st = reinterpret_cast<const uint4*>(stage_base + static_cast<size_t>(s) * kBulkTileBytes);
+        // Reduces the tile in `st` (nv vectors, the row's vectors v0..) into the running candidate; GT threads share it.
+        auto reduce_tile = [&](auto group_threads, const uint4* st, int gt, int v0, int nv, bool row_start) {
+            constexpr int GT = decltype(group_threads)::value;
             int bestq = -1;                                // vector (within this tile) of a new running maximum
 #pragma unroll
-            for (int i = 0; i < kBulkTileVec / kBulkConsumers; ++i) {
-                const int q = ct + i * kBulkConsumers;
+            for (int i = 0; i < kBulkTileVec / GT; ++i) {
+                const int q = gt + i * GT;
                 if (q < nv) {
                     const uint4 v = st[q];
-                    if (i == 0 && ct == 0 && tile == 0) first_nan = rm.v_offset == 0 && bf16_bits_nan(v.x & 0xFFFFu);
+                    if (i == 0 && gt == 0 && row_start) first_nan = rm.v_offset == 0 && bf16_bits_nan(v.x & 0xFFFFu);
                     const float m = vec_max(v);
                     if (m > best) { best = m; bestq = q; }
                 }
@@ -413,20 +445,85 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                 const uint4 v = st[bestq];
                 best_idx = (v0 + bestq) * 8 + first_equal(v, best);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->empty[s]);
-            if (ragged != 0 && tile == tiles_per_row - 1 && ct < ragged) {
-                const int e = nvec_row * 8 + ct;
-                const long long arow = (rm.list != nullptr) ? __ldg(rm.list + row) : row;
-                const unsigned short b = __ldg(reinterpret_cast<const unsigned short*>(logits + arow * stride) + e);
+        };
+        auto ragged_tail = [&](int gt, long long row) {    // the row's last V mod 8 elements, by plain loads
+            if (gt < ragged) {
+                const int e = nvec_row * 8 + gt;
+                const unsigned short b = __ldg(reinterpret_cast<const unsigned short*>(logits + actual_row(row) * stride) + e);
                 const float x = __uint_as_float(static_cast<unsigned>(b) << 16);
-                if (e == 0) first_nan = rm.v_offset == 0 && bf16_bits_nan(b);   // rows shorter than one vector
                 if (x > best) { best = x; best_idx = e; }
             }
-            if (++tile == tiles_per_row) { tile = 0; ++row; }
-            if (++s == kBulkStages) { s = 0; ++use; }
+        };
+
+        if (plan.n_groups == 1) {
+            // ---- large tiles: eight warps take every tile, one after the other
+            if (warp < kWideGroupWarps) {
+                constexpr int GT = kWideGroupWarps * 32;
+                const int ct = threadIdx.x;
+                long long cur_row = -1;
+                long long row = row_first;
+                int tile = static_cast<int>(t0 - row * tiles_per_row);
+                int s = 0;
+                uint32_t use = 0;
+                for (long long t = t0; t < t1; ++t) {
+                    if (row != cur_row) {
+                        if (cur_row >= 0 && !hand_over(static_cast<int>(cur_row - row_first))) { ok = false; break; }
+                        cur_row = row;
+                    }
+                    // the outcome of the wait is made uniform so that the warp leaves the loop together
+                    if (!__all_sync(kFull, mbar_wait_bounded(&sh->full[s], use & 1u, abort))) { ok = false; break; }
+                    const int v0 = tile * tile_vec;
+                    const int nv = max(0, min(tile_vec, nvec_row - v0));
+                    const uint4* st = reinterpret_cast<const uint4*>(stage_base + static_cast<size_t>(s) * plan.stage_bytes);
+                    reduce_tile(std::integral_constant<int, GT>{}, st, ct, v0, nv, tile == 0);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh->empty[s]);
+                    if (ragged != 0 && tile == tiles_per_row - 1) ragged_tail(ct, row);
+                    if (++tile == tiles_per_row) { tile = 0; ++row; }
+                    if (++s == ns) { s = 0; ++use; }
+                }
+                if (ok && cur_row >= 0) ok = hand_over(static_cast<int>(cur_row - row_first));
+            }
+        } else if (warp < n_cons) {
+            // ---- small tiles: groups of four warps take the tiles in turn (tile number `it` of the CTA goes to group
+            // it mod G and sits in stage it mod ns), so that what a tile costs beside its bytes overlaps between groups
+            constexpr int GT = kSmallGroupWarps * 32, G = kSmallGroups;
+            const int group = warp / kSmallGroupWarps;
+            const int gt = threadIdx.x - group * GT;
+            const int stage_bytes = plan.stage_bytes;
+            long long cur_row = row_first;                 // rows before it have been handed over by this warp
+            long long row = row_first;
+            int tile = static_cast<int>(t0 - row * tiles_per_row) + group;
+            while (tile >= tiles_per_row) { tile -= tiles_per_row; ++row; }
+            const int n_tiles_cta = static_cast<int>(t1 - t0);
+            int s = group % ns;                            // stage and use count of the group's next tile, kept incrementally:
+            uint32_t use = static_cast<uint32_t>(group / ns);   // a division per tile would sit on the critical path
+            const unsigned char* stage = stage_base + static_cast<size_t>(s) * stage_bytes;
+            for (int it = group; it < n_tiles_cta && ok; it += G) {
+                while (cur_row < row) {                    // rows finished (or never touched) by this group
+                    if (!hand_over(static_cast<int>(cur_row - row_first))) { ok = false; break; }
+                    ++cur_row;
+                }
+                if (!ok) break;
+                if (!__all_sync(kFull, mbar_wait_bounded(&sh->full[s], use & 1u, abort))) { ok = false; break; }
+                const int v0 = tile * tile_vec;
+                const int nv = max(0, min(tile_vec, nvec_row - v0));
+                reduce_tile(std::integral_constant<int, GT>{}, reinterpret_cast<const uint4*>(stage), gt, v0, nv, tile == 0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->empty[s]);
+                if (ragged != 0 && tile == tiles_per_row - 1) ragged_tail(gt, row);
+                tile += G;
+                while (tile >= tiles_per_row) { tile -= tiles_per_row; ++row; }
+                s += G;                                    // G <= ns
+                stage += static_cast<size_t>(G) * stage_bytes;
+                if (s >= ns) { s -= ns; ++use; stage -= static_cast<size_t>(ns) * stage_bytes; }
+            }
+            // the rest of the CTA's rows (the last one this group worked on, and any behind it)
+            while (ok && cur_row < row_first + n_rows) {
+                ok = hand_over(static_cast<int>(cur_row - row_first));
+                ++cur_row;
+            }
         }
-        if (ok) ok = flush();
         if (!ok && lane == 0) {
             *abort = 1;
             atomicExch(status, kStatusWaitTimeout);
@@ -438,10 +535,10 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         // copies already issued must land before this CTA's shared memory is given up
         if (threadIdx.x == 0) {
             const long long issued = sh->issued;
-            const long long first = (issued > kBulkStages) ? issued - kBulkStages : 0;
+            const long long first = (issued > ns) ? issued - ns : 0;
             for (long long j = first; j < issued; ++j) {
-                const int sj = static_cast<int>(j % kBulkStages);
-                const uint32_t uj = static_cast<uint32_t>(j / kBulkStages);
+                const int sj = static_cast<int>(j % ns);
+                const uint32_t uj = static_cast<uint32_t>(j / ns);
                 int never = 0;
                 mbar_wait_bounded(&sh->full[sj], uj & 1u, &never);
             }

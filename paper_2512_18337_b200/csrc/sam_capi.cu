@@ -89,7 +89,7 @@ inline int* status_word(unsigned long long* keys, int64_t R) {
 // Partial results land in keys[R]; `status` receives a non-zero code if a kernel gives up on an
 // internal wait.
 // Layout of the verification scratch:
-// keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B] | row_list[R] | n_rows (256 B)
+// keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B] | row_list[R] | list meta words (256 B)
 struct Scratch {
     unsigned long long* keys;
     int* status;
@@ -97,7 +97,7 @@ struct Scratch {
     int* pre_len;
     int* done;
     int* row_list;
-    int* n_rows;
+    int* list_meta;
     int64_t bytes;
 };
 Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M: automaton slots per stream (walk-ahead arrays)
@@ -112,7 +112,7 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M
     s.pre_len = reinterpret_cast<int*>(p + o);              o = up(o + static_cast<int64_t>(B) * M * K * 4);
     s.done = reinterpret_cast<int*>(p + o);                 o = up(o + static_cast<int64_t>(B) * 4);
     s.row_list = reinterpret_cast<int*>(p + o);             o = up(o + R * 4);
-    s.n_rows = reinterpret_cast<int*>(p + o);               o += 256;
+    s.list_meta = reinterpret_cast<int*>(p + o);            o += 256;
     s.bytes = o;
     return s;
 }
@@ -137,9 +137,9 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != SAM_OK) return rc;
-    const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0;
+    const bool rows_aligned = aligned(logits, 16) && (stride % 8) == 0 && V >= 8;
     const bool bulk = rows_aligned && g_argmax_variant != 1 && !latency_case;
-    const RowMap rm = rmap ? *rmap : RowMap{nullptr, nullptr, 0};
+    const RowMap rm = rmap ? *rmap : RowMap{nullptr, nullptr, 0, 0, nullptr};
     if (did_prewalk) *did_prewalk = false;
     if (did_tail) *did_tail = false;
     if (bulk) {
@@ -151,9 +151,10 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
                                           static_cast<int>(kBulkSmemBytes)));
             attr_dev = dev;
         }
-        const int64_t nvec = V / 8;
-        const int tiles_per_row = static_cast<int>(nvec > 0 ? (nvec + kBulkTileVec - 1) / kBulkTileVec : 1);
-        const int tile_vec = static_cast<int>(nvec > 0 ? (nvec + tiles_per_row - 1) / tiles_per_row : 1);
+        // a row is cut into the fewest tiles that fit a stage, all nearly equal (large tiles amortise what a tile costs
+        // beside its bytes); the R * tiles_per_row tiles are split into equal contiguous ranges, one persistent CTA per SM
+        const BulkPlan plan = bulk_plan(V);
+        const int tiles_per_row = plan.tiles_per_row;
         const int64_t total = R * tiles_per_row;
         int64_t grid = di.sms;
         if (grid > total) grid = total;
@@ -173,7 +174,7 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
             }
         }
         argmax_bulk_kernel<<<static_cast<unsigned>(grid), kBulkThreads, kBulkSmemBytes, st>>>(
-            static_cast<const __nv_bfloat16*>(logits), stride, R, V, tiles_per_row, tile_vec, keys, status,
+            static_cast<const __nv_bfloat16*>(logits), stride, R, V, plan, keys, status,
             sam ? *sam : DeviceSam{}, pw ? *pw : PreWalk{}, ft, rm);
         ++g_launches;
         if (did_prewalk) *did_prewalk = prewalk;
@@ -249,11 +250,197 @@ int apply_full(sam_index* idx, const Delta& D, cudaStream_t st) {
     return SAM_OK;
 }
 
-constexpr int kDirectRowEdges = 2048;   // rows at least this long are copied straight to their place
+}  // namespace
 
-// Scatters one update through the staging area, in as many rounds as its size needs.  Host buffers are
-// pageable, so every cudaMemcpyAsync has taken its copy of the source when it returns.
-int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st) {
+// ---- small updates sent ahead of time -------------------------------------------------------------
+// The builder thread copies every small update into a slot of the blob's ring as soon as it is packed: through
+// page-locked memory, on a stream of the library's own, while decoding steps run on the caller's stream.  The copy
+// touches nothing that a kernel reads.  sam_sync then only makes the caller's stream wait for the slot's event
+// and launches the one kernel that scatters the slot into the live records - the only work that has to sit between
+// two steps.  A slot is reused once the kernel that read it has finished.
+struct samb200::UpdateRing {
+    int device = -1;
+    cudaStream_t copy_stream = nullptr;
+    char* pinned = nullptr;                       // kRingSlots * kRingSlotBytes, page-locked
+    char* dev_ring = nullptr;                     // the ring inside the caller's blob
+    cudaEvent_t copied[kRingSlots] = {};          // the slot's copy has arrived
+    cudaEvent_t applied[kRingSlots] = {};         // the kernel that read the slot has finished
+    enum : int { kFree = 0, kStaged = 1, kApplied = 2 };
+    int state[kRingSlots] = {};
+    int next = 0;
+    uint64_t epoch = 0;                           // changes with every (re-)upload: slots staged before it are void
+    bool enabled = false;
+    std::mutex mu;
+};
+
+namespace {
+
+void ring_destroy(sam_index* idx) {
+    UpdateRing* r = idx->ring;
+    if (!r) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (r->device >= 0) cudaSetDevice(r->device);
+    if (r->copy_stream) {
+        cudaStreamSynchronize(r->copy_stream);
+        cudaStreamDestroy(r->copy_stream);
+    }
+    for (int k = 0; k < kRingSlots; ++k) {
+        if (r->copied[k]) cudaEventDestroy(r->copied[k]);
+        if (r->applied[k]) { cudaEventSynchronize(r->applied[k]); cudaEventDestroy(r->applied[k]); }
+    }
+    if (r->pinned) cudaFreeHost(r->pinned);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete r;
+    idx->ring = nullptr;
+}
+
+// (Re-)creates the ring for the blob just uploaded; everything staged for an earlier blob is void.  Setup, not hot path.
+int ring_attach(sam_index* idx, char* dev_ring) {
+    UpdateRing* r = idx->ring;
+    if (!r) {
+        r = new (std::nothrow) UpdateRing();
+        if (!r) return SAM_ERR_NOMEM;
+        idx->ring = r;
+    }
+    std::lock_guard<std::mutex> lock(r->mu);
+    r->enabled = false;
+    int dev = 0;
+    SAM_CUDA(cudaGetDevice(&dev));
+    if (r->copy_stream && r->device != dev) return SAM_ERR_INVALID_ARG;      // a handle stays on the device of its first upload
+    r->device = dev;
+    if (!r->copy_stream) {
+        SAM_CUDA(cudaStreamCreateWithFlags(&r->copy_stream, cudaStreamNonBlocking));
+        void* hp = nullptr;
+        SAM_CUDA(cudaHostAlloc(&hp, static_cast<size_t>(kRingSlots * kRingSlotBytes), cudaHostAllocDefault));
+        r->pinned = static_cast<char*>(hp);
+        for (int k = 0; k < kRingSlots; ++k) {
+            SAM_CUDA(cudaEventCreateWithFlags(&r->copied[k], cudaEventDisableTiming));
+            SAM_CUDA(cudaEventCreateWithFlags(&r->applied[k], cudaEventDisableTiming));
+        }
+    } else {
+        SAM_CUDA(cudaStreamSynchronize(r->copy_stream));
+    }
+    for (int k = 0; k < kRingSlots; ++k) r->state[k] = UpdateRing::kFree;
+    r->next = 0;
+    ++r->epoch;
+    r->dev_ring = dev_ring;
+    r->enabled = true;
+    return SAM_OK;
+}
+
+}  // namespace
+
+// Builder thread: the update goes to the next ring slot if it is small enough and a slot is free; otherwise it stays
+// as it is and sam_sync copies it on the caller's stream.
+void samb200::ring_stage_async(sam_index* idx, Delta* D) {
+    UpdateRing* r = idx->ring;
+    if (!r || D->full || D->status != SAM_OK) return;
+    StagedLayout L;
+    staged_layout(*D, &L);
+    if (L.total <= 0 || L.total > kRingSlotBytes) return;
+    int k = -1, was = 0;
+    uint64_t epoch = 0;
+    {
+        std::lock_guard<std::mutex> lock(r->mu);
+        if (!r->enabled || r->state[r->next] == UpdateRing::kStaged) return;     // no blob yet, or sam_sync is 8 updates behind
+        k = r->next;
+        was = r->state[k];
+        r->state[k] = UpdateRing::kStaged;
+        r->next = (k + 1) % kRingSlots;
+        epoch = r->epoch;
+    }
+    static thread_local int dev_set = -1;
+    bool ok = true;
+    if (dev_set != r->device) {
+        ok = cudaSetDevice(r->device) == cudaSuccess;
+        if (ok) dev_set = r->device;
+    }
+    // the kernel that read this slot last (and with it the copy that filled it) must be over
+    if (ok && was == UpdateRing::kApplied) ok = cudaEventSynchronize(r->applied[k]) == cudaSuccess;
+    if (ok) {
+        char* h = r->pinned + k * kRingSlotBytes;
+        staged_fill(*D, L, h);
+        ok = cudaMemcpyAsync(r->dev_ring + k * kRingSlotBytes, h, static_cast<size_t>(L.total), cudaMemcpyHostToDevice,
+                             r->copy_stream) == cudaSuccess &&
+             cudaEventRecord(r->copied[k], r->copy_stream) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        std::lock_guard<std::mutex> lock(r->mu);
+        if (r->epoch == epoch) r->state[k] = UpdateRing::kFree;
+        return;
+    }
+    D->staged_slot = k;
+    D->staged_epoch = epoch;
+    D->staged = L;
+}
+
+namespace {
+
+UpdateArgs update_args(sam_index* idx, const Delta& D, const StagedLayout& L, const char* stage) {
+    const DeviceLayout& dl = idx->layout;
+    char* base = static_cast<char*>(idx->device_buf);
+    UpdateArgs a{};
+    a.rec = reinterpret_cast<StateRec*>(base + dl.rec_off);
+    a.wide = reinterpret_cast<Edge*>(base + dl.edge_off);
+    a.root = reinterpret_cast<int32_t*>(base + dl.root_off);
+    a.corpus = reinterpret_cast<int32_t*>(base + dl.corpus_off) + D.corpus_off;
+    a.stage = stage;
+    a.off_ids = L.off_ids; a.off_recs = L.off_recs; a.off_descs = L.off_descs; a.off_edges = L.off_edges;
+    a.off_rtok = L.off_rtok; a.off_rdst = L.off_rdst; a.off_tail = L.off_tail;
+    a.n_rec = L.n_rec; a.n_seg = L.n_seg; a.n_root = L.n_root; a.n_tail = L.n_tail;
+    a.root_span = static_cast<int>(dl.root_span);
+    return a;
+}
+
+// The stream states to repair after an update (sam_sync_renormalize), or nothing (B = 0).
+struct Renorm {
+    int32_t B = 0;
+    int32_t* state = nullptr;
+    const int32_t* matched_len = nullptr;
+};
+
+// Launches the scatter kernel over a staged buffer; with `rn`, the kernel also repairs the stream states at its end.
+int launch_update_kernel(sam_index* idx, const Delta& D, const StagedLayout& L, const char* stage, const Renorm* rn,
+                         cudaStream_t st) {
+    const UpdateArgs a = update_args(idx, D, L, stage);
+    RenormTail t{};
+    if (rn && rn->B > 0) {
+        t.sam = idx->dev;
+        t.sam.n_states = static_cast<int32_t>(D.n_states_after);       // the view this update leaves behind
+        t.sam.n_corpus = D.n_tokens_after;
+        t.B = rn->B;
+        t.state = rn->state;
+        t.matched_len = rn->matched_len;
+        t.blocks_done = reinterpret_cast<unsigned*>(static_cast<char*>(idx->device_buf) + idx->layout.ctrl_off);
+    }
+    const int64_t work = std::max(std::max<int64_t>(L.n_rec, int64_t(L.n_seg) * 32), std::max<int64_t>(L.n_root, L.n_tail));
+    const unsigned blocks = static_cast<unsigned>(std::min<int64_t>(1184, std::max<int64_t>(1, (work + 255) / 256)));
+    apply_update_kernel<<<blocks, 256, 0, st>>>(a, t);
+    SAM_CUDA(cudaGetLastError());
+    ++g_launches;
+    return SAM_OK;
+}
+
+int copy_long_rows(sam_index* idx, const Delta& D, cudaStream_t st) {
+    Edge* wide = reinterpret_cast<Edge*>(static_cast<char*>(idx->device_buf) + idx->layout.edge_off);
+    for (const WideSeg& g : D.segs)
+        if (g.len >= kDirectRowEdges)
+            SAM_CUDA(cudaMemcpyAsync(wide + g.dst_off, D.seg_edges.data() + g.src_off,
+                                     static_cast<size_t>(g.len) * sizeof(Edge), cudaMemcpyHostToDevice, st));
+    return SAM_OK;
+}
+
+bool has_long_rows(const Delta& D) {
+    for (const WideSeg& g : D.segs)
+        if (g.len >= kDirectRowEdges) return true;
+    return false;
+}
+
+// Scatters one update.  *renormalized tells whether the launch also repaired the stream states of `rn`.
+// Host buffers are pageable, so every cudaMemcpyAsync has taken its copy of the source when it returns.
+int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st, const Renorm* rn, bool* renormalized) {
     const DeviceLayout& L = idx->layout;
     char* base = static_cast<char*>(idx->device_buf);
     char* stage = base + L.stage_off;
@@ -261,74 +448,63 @@ int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st) {
     Edge* wide = reinterpret_cast<Edge*>(base + L.edge_off);
     int32_t* root = reinterpret_cast<int32_t*>(base + L.root_off);
     const int64_t n_rec = static_cast<int64_t>(D.rec_ids.size());
-    // ---- small update (the usual case between two decoding steps): everything but rows long enough to be copied
-    // on their own goes through one page-locked buffer, one copy and one kernel
+    *renormalized = false;
+    // rows long enough to be copied on their own must be in place before the states are repaired
+    const Renorm* tail = (rn && rn->B > 0 && !has_long_rows(D)) ? rn : nullptr;
+    // ---- already on the device: the builder thread sent it to a ring slot
+    UpdateRing* r = idx->ring;
+    if (D.staged_slot >= 0 && r) {
+        bool valid;
+        {
+            std::lock_guard<std::mutex> lock(r->mu);
+            valid = r->enabled && r->epoch == D.staged_epoch;
+        }
+        if (valid) {
+            const int k = D.staged_slot;
+            // normally the copy arrived long ago; only if it has not does the caller's stream have to wait for it
+            if (cudaEventQuery(r->copied[k]) != cudaSuccess) {
+                cudaGetLastError();
+                SAM_CUDA(cudaStreamWaitEvent(st, r->copied[k], 0));
+            }
+            int rc = launch_update_kernel(idx, D, D.staged, r->dev_ring + k * kRingSlotBytes, tail, st);
+            if (rc != SAM_OK) return rc;
+            SAM_CUDA(cudaEventRecord(r->applied[k], st));
+            {
+                std::lock_guard<std::mutex> lock(r->mu);
+                if (r->epoch == D.staged_epoch) r->state[k] = UpdateRing::kApplied;
+            }
+            *renormalized = tail != nullptr;
+            return copy_long_rows(idx, D, st);
+        }
+    }
+    // ---- small update that was not sent ahead: one page-locked buffer, one copy and one kernel on the caller's stream
     {
-        constexpr int64_t kPinnedBytes = int64_t(1) << 20;
-        auto up32 = [](int64_t x) { return (x + 31) & ~int64_t(31); };
-        int64_t n_seg = 0, n_edges = 0;
-        for (const WideSeg& g : D.segs)
-            if (g.len < kDirectRowEdges) { ++n_seg; n_edges += g.len; }
-        const int64_t n_root = static_cast<int64_t>(D.root_tok.size());
-        const int64_t n_tail = static_cast<int64_t>(D.corpus_tail.size());
-        UpdateArgs a{};
-        a.off_ids = 0;
-        a.off_recs = up32(n_rec * 4);
-        a.off_descs = a.off_recs + n_rec * static_cast<int64_t>(sizeof(StateRec));
-        a.off_edges = up32(a.off_descs + n_seg * static_cast<int64_t>(sizeof(SegDesc)));
-        a.off_rtok = up32(a.off_edges + n_edges * static_cast<int64_t>(sizeof(Edge)));
-        a.off_rdst = up32(a.off_rtok + n_root * 4);
-        a.off_tail = up32(a.off_rdst + n_root * 4);
-        const int64_t total = up32(a.off_tail + n_tail * 4);
-        if (total <= kPinnedBytes && total <= L.stage_bytes) {
+        StagedLayout a;
+        staged_layout(D, &a);
+        if (a.total <= kRingSlotBytes && a.total <= L.stage_bytes) {
             if (!idx->pinned_stage) {
                 void* hp = nullptr;
                 cudaEvent_t ev = nullptr;
-                SAM_CUDA(cudaHostAlloc(&hp, static_cast<size_t>(kPinnedBytes), cudaHostAllocDefault));
+                SAM_CUDA(cudaHostAlloc(&hp, static_cast<size_t>(kRingSlotBytes), cudaHostAllocDefault));
                 const cudaError_t e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
                 if (e != cudaSuccess) { cudaFreeHost(hp); return cuda_fail(e); }
                 idx->pinned_stage = hp;
-                idx->pinned_bytes = kPinnedBytes;
+                idx->pinned_bytes = kRingSlotBytes;
                 idx->stage_event = ev;
             } else {
                 // the previous update's copy must have left the buffer before it is refilled
                 SAM_CUDA(cudaEventSynchronize(static_cast<cudaEvent_t>(idx->stage_event)));
             }
             char* h = static_cast<char*>(idx->pinned_stage);
-            std::memcpy(h + a.off_ids, D.rec_ids.data(), static_cast<size_t>(n_rec) * 4);
-            std::memcpy(h + a.off_recs, D.recs.data(), static_cast<size_t>(n_rec) * sizeof(StateRec));
-            SegDesc* descs = reinterpret_cast<SegDesc*>(h + a.off_descs);
-            Edge* edges = reinterpret_cast<Edge*>(h + a.off_edges);
-            int64_t ns = 0, ne = 0;
-            for (const WideSeg& g : D.segs) {
-                if (g.len >= kDirectRowEdges) continue;
-                descs[ns++] = SegDesc{g.dst_off, static_cast<int>(ne), g.len};
-                std::memcpy(edges + ne, D.seg_edges.data() + g.src_off, static_cast<size_t>(g.len) * sizeof(Edge));
-                ne += g.len;
-            }
-            std::memcpy(h + a.off_rtok, D.root_tok.data(), static_cast<size_t>(n_root) * 4);
-            std::memcpy(h + a.off_rdst, D.root_dst.data(), static_cast<size_t>(n_root) * 4);
-            std::memcpy(h + a.off_tail, D.corpus_tail.data(), static_cast<size_t>(n_tail) * 4);
-            if (total > 0) {
-                SAM_CUDA(cudaMemcpyAsync(stage, h, static_cast<size_t>(total), cudaMemcpyHostToDevice, st));
+            staged_fill(D, a, h);
+            if (a.total > 0) {
+                SAM_CUDA(cudaMemcpyAsync(stage, h, static_cast<size_t>(a.total), cudaMemcpyHostToDevice, st));
                 SAM_CUDA(cudaEventRecord(static_cast<cudaEvent_t>(idx->stage_event), st));
-                a.rec = rec; a.wide = wide; a.root = root;
-                a.corpus = reinterpret_cast<int32_t*>(base + L.corpus_off) + D.corpus_off;
-                a.stage = stage;
-                a.n_rec = static_cast<int>(n_rec); a.n_seg = static_cast<int>(n_seg);
-                a.n_root = static_cast<int>(n_root); a.n_tail = static_cast<int>(n_tail);
-                a.root_span = static_cast<int>(L.root_span);
-                const int64_t work = std::max(std::max(n_rec, n_seg * 32), std::max(n_root, n_tail));
-                const unsigned blocks = static_cast<unsigned>(std::min<int64_t>(1184, std::max<int64_t>(1, (work + 255) / 256)));
-                apply_update_kernel<<<blocks, 256, 0, st>>>(a);
-                SAM_CUDA(cudaGetLastError());
-                ++g_launches;
+                const int rc = launch_update_kernel(idx, D, a, stage, tail, st);
+                if (rc != SAM_OK) return rc;
+                *renormalized = tail != nullptr;
             }
-            for (const WideSeg& g : D.segs)
-                if (g.len >= kDirectRowEdges)
-                    SAM_CUDA(cudaMemcpyAsync(wide + g.dst_off, D.seg_edges.data() + g.src_off,
-                                             static_cast<size_t>(g.len) * sizeof(Edge), cudaMemcpyHostToDevice, st));
-            return SAM_OK;
+            return copy_long_rows(idx, D, st);
         }
     }
     // ---- large update: section by section through the staging area
@@ -408,9 +584,11 @@ int apply_changes(sam_index* idx, const Delta& D, cudaStream_t st) {
     return SAM_OK;
 }
 
-int apply_delta(sam_index* idx, const Delta& D, cudaStream_t st) {
+int apply_delta(sam_index* idx, const Delta& D, cudaStream_t st, const Renorm* rn = nullptr, bool* renormalized = nullptr) {
     if (D.status != SAM_OK) return D.status;
-    const int rc = D.full ? apply_full(idx, D, st) : apply_changes(idx, D, st);
+    bool did = false;
+    const int rc = D.full ? apply_full(idx, D, st) : apply_changes(idx, D, st, rn, &did);
+    if (renormalized) *renormalized = did;
     if (rc != SAM_OK) return rc;
     idx->dev.n_states = static_cast<int32_t>(D.n_states_after);
     idx->dev.n_corpus = D.n_tokens_after;
@@ -420,6 +598,10 @@ int apply_delta(sam_index* idx, const Delta& D, cudaStream_t st) {
 }
 
 int upload_growing(sam_index* idx, void* device_buf, cudaStream_t st) {
+    if (idx->ring) {       // nothing more is sent towards the blob that is being replaced
+        std::lock_guard<std::mutex> lock(idx->ring->mu);
+        idx->ring->enabled = false;
+    }
     Delta image;
     int rc = dyn_full_image(idx, &image);
     if (rc != SAM_OK) return rc;
@@ -430,7 +612,45 @@ int upload_growing(sam_index* idx, void* device_buf, cudaStream_t st) {
         idx->device_buf = nullptr;
         return rc;
     }
+    char* base = static_cast<char*>(device_buf);
+    SAM_CUDA(cudaMemsetAsync(base + idx->layout.ctrl_off, 0, 256, st));
     SAM_CUDA(cudaStreamSynchronize(st));
+    return ring_attach(idx, base + idx->layout.ring_off);
+}
+
+// sam_sync with or without the repair of stream states at the end of the last update's kernel.
+int sync_updates(sam_index* idx, cudaStream_t st, const Renorm* rn, int64_t* tokens_on_device) {
+    std::vector<Delta> ready;
+    {
+        Delta D;
+        while (dyn_pop_ready(idx, &D)) ready.push_back(std::move(D));
+    }
+    bool repaired = ready.empty();         // nothing changed: nothing to repair
+    for (size_t i = 0; i < ready.size(); ++i) {
+        const Delta& D = ready[i];
+        const bool last = i + 1 == ready.size();
+        bool did = false;
+        const int rc = apply_delta(idx, D, st, last ? rn : nullptr, &did);
+        if (rc != SAM_OK) return rc;
+        if (last) repaired = did;
+        if (D.full) {
+            ++idx->updates_full;
+            idx->update_bytes += static_cast<int64_t>(D.all_rec.size() * sizeof(StateRec) + D.all_wide.size() * sizeof(Edge) +
+                                                      (D.all_root.size() + D.all_corpus.size()) * 4);
+        } else {
+            ++idx->updates_incremental;
+            idx->update_bytes += static_cast<int64_t>(D.rec_ids.size() * 36 + D.seg_edges.size() * sizeof(Edge) +
+                                                      D.segs.size() * sizeof(SegDesc) + D.root_tok.size() * 8 +
+                                                      D.corpus_tail.size() * 4);
+        }
+    }
+    if (rn && rn->B > 0 && !repaired) {
+        // the last update went section by section (or was a whole image): the states are repaired by a kernel of their own
+        renormalize_kernel<<<static_cast<unsigned>((rn->B + 127) / 128), 128, 0, st>>>(idx->dev, rn->B, rn->state, rn->matched_len);
+        SAM_CUDA(cudaGetLastError());
+        ++g_launches;
+    }
+    if (tokens_on_device) *tokens_on_device = idx->dev.n_corpus;
     return SAM_OK;
 }
 
@@ -535,7 +755,8 @@ void sam_free(sam_index* idx) {
         cudaEventDestroy(static_cast<cudaEvent_t>(idx->stage_event));
     }
     if (idx->pinned_stage) cudaFreeHost(idx->pinned_stage);
-    dyn_destroy(idx);
+    dyn_destroy(idx);          // joins the builder thread, which may be sending an update to the ring
+    ring_destroy(idx);
     delete idx;
 }
 
@@ -582,13 +803,12 @@ int sam_verify_ex(const void* logits_bf16, int64_t row_stride_elems, int32_t B, 
     const AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
                         argmax_out, accepted, n_accepted, sc.keys, nullptr, nullptr, 1, nullptr, nullptr,
                         nullptr, nullptr, flags, reinterpret_cast<unsigned long long*>(counters)};
-    RowMap rm{nullptr, nullptr, 0};
+    RowMap rm{nullptr, nullptr, 0, 0, nullptr};
     if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
-        build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.n_rows);
+        build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.list_meta);
         SAM_CUDA(cudaGetLastError());
         ++g_launches;
-        rm.list = sc.row_list;
-        rm.n_rows = sc.n_rows;
+        rm = RowMap{sc.row_list, sc.list_meta, 0, row_list_sig(B, K), sc.status};
     }
     bool did_tail = false;
     rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, nullptr, nullptr, nullptr,
@@ -620,7 +840,9 @@ int sam_step_ex(const sam_index* idx,
                 uint32_t flags, int64_t* counters,
                 void* workspace, int64_t workspace_bytes, void* cuda_stream) {
     if (!idx || min_match < 1) return SAM_ERR_INVALID_ARG;
-    if (flags & ~static_cast<uint32_t>(SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS)) return SAM_ERR_INVALID_ARG;
+    if (flags & ~static_cast<uint32_t>(SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS | SAM_STEP_ROW_LIST_READY))
+        return SAM_ERR_INVALID_ARG;
+    if ((flags & SAM_STEP_ROW_LIST_READY) && !(flags & SAM_STEP_SKIP_UNUSED_ROWS)) return SAM_ERR_INVALID_ARG;
     if (counters && !aligned(counters, 8)) return SAM_ERR_INVALID_ARG;
     int rc = check_verify_args(logits_bf16, row_stride_elems, B, K, V, drafts, n_draft, argmax_out, accepted,
                                n_accepted, workspace, workspace_bytes);
@@ -635,14 +857,21 @@ int sam_step_ex(const sam_index* idx,
                (flags & SAM_STEP_NO_SPECULATION) ? 1 : 0};
     AcceptArgs aa{static_cast<const __nv_bfloat16*>(logits_bf16), row_stride_elems, B, K, drafts, n_draft,
                   argmax_out, accepted, n_accepted, sc.keys, state, matched_len, min_match, next_drafts,
-                  next_n_draft, sc.pre_state, sc.pre_len, flags, reinterpret_cast<unsigned long long*>(counters)};
-    RowMap rm{nullptr, nullptr, 0};
+                  next_n_draft, sc.pre_state, sc.pre_len, flags & (SAM_STEP_NO_SPECULATION | SAM_STEP_SKIP_UNUSED_ROWS),
+                  reinterpret_cast<unsigned long long*>(counters), nullptr, nullptr};
+    RowMap rm{nullptr, nullptr, 0, 0, nullptr};
     if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
-        build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.n_rows);
-        SAM_CUDA(cudaGetLastError());
-        ++g_launches;
-        rm.list = sc.row_list;
-        rm.n_rows = sc.n_rows;
+        // the rows this step reads: listed by the previous step's accept kernel when the caller says so, else by a
+        // small kernel in front; either way this step's accept kernel lists the rows of the next step
+        // (with speculation off for this call the rows wanted are fewer than the previous step listed: list them afresh)
+        if (!(flags & SAM_STEP_ROW_LIST_READY) || (flags & SAM_STEP_NO_SPECULATION)) {
+            build_row_list_kernel<<<1, 1024, 0, st>>>(n_draft, B, K, flags, sc.row_list, sc.list_meta);
+            SAM_CUDA(cudaGetLastError());
+            ++g_launches;
+        }
+        rm = RowMap{sc.row_list, sc.list_meta, 0, row_list_sig(B, K), sc.status};
+        aa.next_list = sc.row_list;
+        aa.list_meta = sc.list_meta;
     }
     bool did_prewalk = false, did_tail = false;
     rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, &idx->dev, &pw, &did_prewalk,
@@ -677,7 +906,7 @@ int sam_argmax_partial(const void* logits_bf16, int64_t row_stride_elems, int64_
     if (!logits_bf16 || !keys || !aligned(logits_bf16, 2) || !aligned(keys, 8)) return SAM_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     SAM_CUDA(cudaMemsetAsync(keys, 0, static_cast<size_t>(rows + 1) * 8, st));     // the last word is the status word
-    const RowMap rm{nullptr, nullptr, v_offset};
+    const RowMap rm{nullptr, nullptr, v_offset, 0, nullptr};
     return launch_argmax(logits_bf16, row_stride_elems, rows, V, reinterpret_cast<unsigned long long*>(keys),
                          reinterpret_cast<int*>(keys + rows), st, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, &rm);
 }
@@ -837,6 +1066,17 @@ int sam_adaptive_switch(int64_t context_len, int64_t batch_size, int64_t max_con
     return (context_len > max_context_len || batch_size > max_batch_size) ? 0 : 1;
 }
 
+int sam_speculation_pays(const int64_t* counters, int32_t K, double cost_ratio) {
+    if (!counters || K < 1 || K > SAM_K_MAX || !(cost_ratio > 0.0)) return SAM_ERR_INVALID_ARG;
+    const int64_t passes = counters[0], accepted_drafts = counters[3], rows_read = counters[5];
+    if (passes < 0 || accepted_drafts < 0 || rows_read < passes) return SAM_ERR_INVALID_ARG;
+    if (passes == 0) return 1;                       // an empty window is no evidence against speculating
+    // tokens gained over plain decoding, scaled by K, against the extra rows read, priced at (cost_ratio - 1) / K each
+    const double gain = static_cast<double>(accepted_drafts) * static_cast<double>(K);
+    const double extra_cost = (cost_ratio - 1.0) * static_cast<double>(rows_read - passes);
+    return gain > extra_cost ? 1 : 0;
+}
+
 namespace {
 struct HostStepLayout {
     int64_t logits, drafts, n_draft, argmax, accepted, n_accepted, state, mlen, ws, total;
@@ -967,15 +1207,30 @@ int sam_step_host_ex(const sam_index* idx,
     char* d = static_cast<char*>(staging);
     const size_t bB = static_cast<size_t>(B) * 4, bK = bB * K, bR = bB * (K + 1);
     if (flags & SAM_STEP_SKIP_UNUSED_ROWS) {
-        // only the rows the step will read cross the bus: rows 0..n_draft[b] of every stream, one copy per stream
+        // only the rows the step will read cross the bus: rows 0..n_draft[b] of every stream.  Runs of rows that touch
+        // (a full proposal is followed directly by the next stream's rows) or that are less than a row apart go in one
+        // copy - a copy costs a few microseconds of its own, about what a row takes on the bus
         const char* src = static_cast<const char*>(logits_bf16);
+        const int64_t row_bytes = row_stride_elems * 2;
+        int64_t run_first = -1, run_end = 0;            // byte range [run_first, run_end) waiting to be copied
         for (int32_t b = 0; b < B; ++b) {
             int32_t nd = (flags & SAM_STEP_NO_SPECULATION) ? 0 : n_draft[b];
             nd = nd < 0 ? 0 : (nd > K ? K : nd);
-            const int64_t first = static_cast<int64_t>(b) * (K + 1) * row_stride_elems * 2;
-            const int64_t bytes = (static_cast<int64_t>(nd) * row_stride_elems + V) * 2;
-            SAM_CUDA(cudaMemcpyAsync(d + L.logits + first, src + first, static_cast<size_t>(bytes), cudaMemcpyHostToDevice, st));
+            const int64_t first = static_cast<int64_t>(b) * (K + 1) * row_bytes;
+            const int64_t end = first + static_cast<int64_t>(nd) * row_bytes + static_cast<int64_t>(V) * 2;
+            if (run_first >= 0 && first - run_end <= row_bytes) {
+                run_end = end;
+                continue;
+            }
+            if (run_first >= 0)
+                SAM_CUDA(cudaMemcpyAsync(d + L.logits + run_first, src + run_first, static_cast<size_t>(run_end - run_first),
+                                         cudaMemcpyHostToDevice, st));
+            run_first = first;
+            run_end = end;
         }
+        if (run_first >= 0)
+            SAM_CUDA(cudaMemcpyAsync(d + L.logits + run_first, src + run_first, static_cast<size_t>(run_end - run_first),
+                                     cudaMemcpyHostToDevice, st));
     } else {
         SAM_CUDA(cudaMemcpyAsync(d + L.logits, logits_bf16, static_cast<size_t>(L.logits_bytes), cudaMemcpyHostToDevice, st));
     }
@@ -1043,24 +1298,16 @@ int sam_pending(sam_index* idx, int64_t* tokens_queued, int64_t* tokens_built, i
 int sam_sync(sam_index* idx, void* cuda_stream, int64_t* tokens_on_device) {
     if (!idx || !idx->dyn) return SAM_ERR_INVALID_ARG;
     if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    Delta D;
-    while (dyn_pop_ready(idx, &D)) {
-        const int rc = apply_delta(idx, D, st);
-        if (rc != SAM_OK) return rc;
-        if (D.full) {
-            ++idx->updates_full;
-            idx->update_bytes += static_cast<int64_t>(D.all_rec.size() * sizeof(StateRec) + D.all_wide.size() * sizeof(Edge) +
-                                                      (D.all_root.size() + D.all_corpus.size()) * 4);
-        } else {
-            ++idx->updates_incremental;
-            idx->update_bytes += static_cast<int64_t>(D.rec_ids.size() * 36 + D.seg_edges.size() * sizeof(Edge) +
-                                                      D.segs.size() * sizeof(SegDesc) + D.root_tok.size() * 8 +
-                                                      D.corpus_tail.size() * 4);
-        }
-    }
-    if (tokens_on_device) *tokens_on_device = idx->dev.n_corpus;
-    return SAM_OK;
+    return sync_updates(idx, static_cast<cudaStream_t>(cuda_stream), nullptr, tokens_on_device);
+}
+
+int sam_sync_renormalize(sam_index* idx, int32_t B, int32_t* state, const int32_t* matched_len, void* cuda_stream,
+                         int64_t* tokens_on_device) {
+    if (!idx || !idx->dyn || B < 0) return SAM_ERR_INVALID_ARG;
+    if (!idx->device_buf) return SAM_ERR_NOT_UPLOADED;
+    if (B > 0 && (!state || !matched_len)) return SAM_ERR_INVALID_ARG;
+    const Renorm rn{B, state, matched_len};
+    return sync_updates(idx, static_cast<cudaStream_t>(cuda_stream), &rn, tokens_on_device);
 }
 
 int sam_update_stats(const sam_index* idx, int64_t* incremental, int64_t* full_images, int64_t* bytes_copied) {

@@ -27,6 +27,7 @@
 namespace samb200 {
 
 struct DynIndex {
+    sam_index* owner = nullptr;
     Builder b;
     int32_t last = 0;
     std::vector<int32_t> corpus;
@@ -300,6 +301,7 @@ void worker_main(DynIndex* D) {
             rc = SAM_ERR_NOMEM;
         }
         delta.status = rc;
+        if (rc == SAM_OK && D->owner) ring_stage_async(D->owner, &delta);   // on its way to the device before anyone asks
         {
             std::lock_guard<std::mutex> lk(D->mu);
             if (rc != SAM_OK) D->error = rc;
@@ -322,6 +324,7 @@ int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tok
     DynIndex* D = nullptr;
     try {
         D = new DynIndex();
+        D->owner = idx;
         D->max_tokens = max_tokens;
         D->s_cap = 2 * max_tokens + 2;
         // sorted rows sit in power-of-two slots (less than twice their length), hash rows are between an eighth
@@ -356,7 +359,9 @@ int dyn_create(sam_index* idx, const int32_t* corpus, int64_t n, int64_t max_tok
     L.root_off = up(L.edge_off + D->w_cap * static_cast<int64_t>(sizeof(Edge)));
     L.corpus_off = up(L.root_off + D->span_cap * 4);
     L.stage_off = up(L.corpus_off + max_tokens * 4);
-    L.total = up(L.stage_off + L.stage_bytes);
+    L.ring_off = up(L.stage_off + L.stage_bytes);
+    L.ctrl_off = up(L.ring_off + kRingSlots * kRingSlotBytes);
+    L.total = up(L.ctrl_off + 256);
     idx->dyn = D;
     D->worker = std::thread(worker_main, D);
     return SAM_OK;
@@ -467,6 +472,49 @@ int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges) {
     if (n_states) *n_states = static_cast<int64_t>(D->b.len.size());
     if (n_edges) *n_edges = static_cast<int64_t>(D->b.e_tok.size());
     return SAM_OK;
+}
+
+void staged_layout(const Delta& D, StagedLayout* out) {
+    auto up32 = [](int64_t x) { return (x + 31) & ~int64_t(31); };
+    int64_t n_seg = 0, n_edges = 0;
+    for (const WideSeg& g : D.segs)
+        if (g.len < kDirectRowEdges) { ++n_seg; n_edges += g.len; }
+    const int64_t n_rec = static_cast<int64_t>(D.rec_ids.size());
+    const int64_t n_root = static_cast<int64_t>(D.root_tok.size());
+    const int64_t n_tail = static_cast<int64_t>(D.corpus_tail.size());
+    StagedLayout& a = *out;
+    a.off_ids = 0;
+    a.off_recs = up32(n_rec * 4);
+    a.off_descs = a.off_recs + n_rec * static_cast<int64_t>(sizeof(StateRec));
+    a.off_edges = up32(a.off_descs + n_seg * 16);
+    a.off_rtok = up32(a.off_edges + n_edges * static_cast<int64_t>(sizeof(Edge)));
+    a.off_rdst = up32(a.off_rtok + n_root * 4);
+    a.off_tail = up32(a.off_rdst + n_root * 4);
+    a.total = up32(a.off_tail + n_tail * 4);
+    a.n_rec = static_cast<int32_t>(n_rec);
+    a.n_seg = static_cast<int32_t>(n_seg);
+    a.n_root = static_cast<int32_t>(n_root);
+    a.n_tail = static_cast<int32_t>(n_tail);
+}
+
+void staged_fill(const Delta& D, const StagedLayout& a, char* h) {
+    // row descriptor as the device reads it: {int64 first edge in the wide array, int32 first edge in the list, int32 length}
+    struct Desc { long long dst_off; int src_off; int len; };
+    static_assert(sizeof(Desc) == 16, "row descriptor");
+    std::memcpy(h + a.off_ids, D.rec_ids.data(), static_cast<size_t>(a.n_rec) * 4);
+    std::memcpy(h + a.off_recs, D.recs.data(), static_cast<size_t>(a.n_rec) * sizeof(StateRec));
+    Desc* descs = reinterpret_cast<Desc*>(h + a.off_descs);
+    Edge* edges = reinterpret_cast<Edge*>(h + a.off_edges);
+    int64_t ns = 0, ne = 0;
+    for (const WideSeg& g : D.segs) {
+        if (g.len >= kDirectRowEdges) continue;
+        descs[ns++] = Desc{g.dst_off, static_cast<int>(ne), g.len};
+        std::memcpy(edges + ne, D.seg_edges.data() + g.src_off, static_cast<size_t>(g.len) * sizeof(Edge));
+        ne += g.len;
+    }
+    std::memcpy(h + a.off_rtok, D.root_tok.data(), static_cast<size_t>(a.n_root) * 4);
+    std::memcpy(h + a.off_rdst, D.root_dst.data(), static_cast<size_t>(a.n_root) * 4);
+    std::memcpy(h + a.off_tail, D.corpus_tail.data(), static_cast<size_t>(a.n_tail) * 4);
 }
 
 int dyn_set_relayout_every(sam_index* idx, int64_t every) {

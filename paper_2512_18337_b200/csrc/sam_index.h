@@ -51,7 +51,18 @@ SAM_HD int32_t hash_log2cap(int32_t deg, int32_t room) {
 struct DeviceLayout {
     int64_t rec_off = 0, edge_off = 0, root_off = 0, corpus_off = 0, stage_off = 0, total = 0;
     int64_t n_states = 0, n_wide_edges = 0, root_span = 0, n_corpus = 0, stage_bytes = 0;
+    int64_t ring_off = 0, ctrl_off = 0;      // growing index: slots for updates copied ahead of time; a few control words
 };
+
+// Updates of a growing index that are small enough (the usual case between two decoding steps) travel as one flat
+// buffer: [record ids][records][row descriptors][row edges][root tokens][root destinations][appended text].
+struct StagedLayout {
+    int64_t off_ids = 0, off_recs = 0, off_descs = 0, off_edges = 0, off_rtok = 0, off_rdst = 0, off_tail = 0, total = 0;
+    int32_t n_rec = 0, n_seg = 0, n_root = 0, n_tail = 0;
+};
+constexpr int kRingSlots = 8;                          // updates that can wait on the device for sam_sync
+constexpr int64_t kRingSlotBytes = int64_t(1) << 20;   // largest update that takes this route
+constexpr int kDirectRowEdges = 2048;                  // rows at least this long are copied straight to their place
 
 // Pointers handed to kernels by value.
 struct DeviceSam {
@@ -85,12 +96,17 @@ struct Delta {
     int64_t corpus_off = 0;                  // appended text
     std::vector<int32_t> corpus_tail;
     int64_t n_states_after = 0, n_tokens_after = 0;
+    // set by the builder thread when it has already sent the update to a ring slot of the device blob
+    int staged_slot = -1;
+    uint64_t staged_epoch = 0;
+    StagedLayout staged;
     // full image only
     std::vector<StateRec> all_rec;
     std::vector<Edge> all_wide;
     std::vector<int32_t> all_root, all_corpus;
 };
 struct DynIndex;   // host-side state of a growing index (sam_dynamic.cpp)
+struct UpdateRing; // CUDA objects of the asynchronous update path (sam_capi.cu)
 
 }  // namespace samb200
 
@@ -113,6 +129,8 @@ struct sam_index {
     void* pinned_stage = nullptr;
     int64_t pinned_bytes = 0;
     void* stage_event = nullptr;
+    // copy stream, page-locked slots and events with which the builder thread sends small updates ahead of sam_sync
+    samb200::UpdateRing* ring = nullptr;
 };
 
 namespace samb200 {
@@ -131,5 +149,10 @@ int dyn_full_image(sam_index* idx, Delta* out);                        // waits,
 int dyn_sizes(sam_index* idx, int64_t* n_states, int64_t* n_edges);    // waits; states / transitions right now
 int dyn_refresh_csr(sam_index* idx);                                   // waits, refills the flat arrays for sam_export
 void dyn_counts(sam_index* idx, int64_t* queued, int64_t* built);      // tokens handed in / tokens indexed on the host
-int dyn_set_relayout_every(sam_index* idx, int64_t every);             // every k-th update becomes a whole image (0: never forced)
+int dyn_set_relayout_every(sam_index* idx, int64_t every);
+// Layout of a small update's flat buffer, and the buffer itself (h holds layout.total bytes).
+void staged_layout(const Delta& D, StagedLayout* out);
+void staged_fill(const Delta& D, const StagedLayout& L, char* h);
+// Called by the builder thread for every finished update: copies it towards the device if it can (sam_capi.cu).
+void ring_stage_async(sam_index* idx, Delta* D);             // every k-th update becomes a whole image (0: never forced)
 }  // namespace samb200

@@ -380,24 +380,45 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+// Status word of the verification scratch (sam_workspace_status).
+enum : int { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusQueueOverflow = 2, kStatusBadRowList = 3 };
+
 // Optional indirection and offset for the argmax kernels.
-//   list / n_rows: only the rows list[0..*n_rows) are reduced, in that order (both in device memory);
-//                  nullptr: all rows 0..R-1.
+//   list / meta:   only the rows list[0..meta[kListCount]) are reduced, in that order (both in device memory);
+//                  the list counts only if meta[kListSig] == sig (it was made for this batch shape), otherwise
+//                  nothing is reduced and *status is raised.  list == nullptr: all rows 0..R-1.
 //   v_offset:      added to every index (the logits are columns v_offset.. of a wider vocabulary).
+// meta words: [kListCount] rows in the list; [kListAccum] rows collected so far for the NEXT list (zero between
+// calls); [kListArrived] streams that have added theirs (zero between calls); [kListSig] shape the list was made for.
+enum : int { kListCount = 0, kListAccum = 1, kListArrived = 2, kListSig = 3 };
 struct RowMap {
     const int* list;
-    const int* n_rows;
+    const int* meta;
     int v_offset;
+    int sig;
+    int* status;
 };
+__host__ __device__ __forceinline__ int row_list_sig(int B, int K) {
+    return static_cast<int>((static_cast<unsigned>(B) << 6) ^ static_cast<unsigned>(K) ^ 0x5A000000u);
+}
+// Rows the list holds for this call (0 and a raised status word when the list is not one for this call).
+__device__ __forceinline__ long long listed_rows(const RowMap& rm, long long R) {
+    const long long n = __ldg(rm.meta + kListCount);
+    if (__ldg(rm.meta + kListSig) != rm.sig || n < 0 || n > R) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicExch(rm.status, kStatusBadRowList);
+        return 0;
+    }
+    return n;
+}
 
 // Step options (same values as SAM_STEP_* in sam.h).
-constexpr unsigned kNoSpeculation = 1u, kSkipUnusedRows = 2u;
+constexpr unsigned kNoSpeculation = 1u, kSkipUnusedRows = 2u, kRowListReady = 4u;
 
 // Rows 0..n_draft[b] of every stream, in stream order (n_draft clamped to 0..K, or 0 when speculation
-// is off); one CTA, a block-wide running sum.  *n_rows receives the count.
+// is off); one CTA, a block-wide running sum.  meta receives the count and the shape signature.
 __global__ void __launch_bounds__(1024)
 build_row_list_kernel(const int* __restrict__ n_draft, int B, int K, unsigned flags,
-                      int* __restrict__ list, int* __restrict__ n_rows) {
+                      int* __restrict__ list, int* __restrict__ meta) {
     __shared__ int warp_sum[32];
     __shared__ int carry;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -423,7 +444,10 @@ build_row_list_kernel(const int* __restrict__ n_draft, int B, int K, unsigned fl
         if (threadIdx.x == blockDim.x - 1) carry = before + incl;
         __syncthreads();
     }
-    if (threadIdx.x == 0) *n_rows = carry;
+    if (threadIdx.x == 0) {
+        meta[kListCount] = carry;
+        meta[kListSig] = row_list_sig(B, K);
+    }
 }
 
 constexpr int kArgmaxThreads = 256;
@@ -462,7 +486,8 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
                      int tiles_per_row, unsigned long long* __restrict__ keys, RowMap rm) {
     // the accept kernel may be scheduled now; it waits for this grid before it reads any result
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (rm.list != nullptr) R = __ldg(rm.n_rows);
+    const long long R_all = R;
+    if (rm.list != nullptr) R = listed_rows(rm, R_all);
     const long long total = R * tiles_per_row;
     const long long t0 = total * blockIdx.x / gridDim.x;
     const long long t1 = total * (blockIdx.x + 1) / gridDim.x;
@@ -490,7 +515,11 @@ argmax_direct_kernel(const __nv_bfloat16* __restrict__ logits, long long stride,
     for (long long t = t0; t < t1; ++t) {
         const long long vrow = t / tiles_per_row;
         const int tile = static_cast<int>(t - vrow * tiles_per_row);
-        const long long row = (rm.list != nullptr) ? __ldg(rm.list + vrow) : vrow;
+        long long row = vrow;
+        if (rm.list != nullptr) {              // clamped: a foreign list can give wrong results, never a fault
+            row = __ldg(rm.list + vrow);
+            row = row < 0 ? 0 : (row >= R_all ? R_all - 1 : row);
+        }
         if (row != cur_row) {
             flush();
             cur_row = row;
@@ -552,6 +581,8 @@ struct AcceptArgs {
     const int* pre_len;       // [B, K]
     unsigned flags;           // kNoSpeculation | kSkipUnusedRows
     unsigned long long* counters;   // [6] running statistics, or nullptr
+    int* next_list;           // row list of the NEXT step (rows 0..next_n_draft[b] of every stream, any order), or nullptr
+    int* list_meta;           // its meta words (see RowMap)
 };
 
 // One warp, one stream.  The packed candidates and the walk-ahead results may have been produced
@@ -665,6 +696,26 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
             p.state[b] = s;
             p.matched_len[b] = L;
             p.next_n_draft[b] = nn;
+        }
+        if (p.next_list != nullptr) {
+            // The rows the next step will need from this stream go into the next row list.  The argmax kernel that
+            // read the current list has finished (this kernel waited for it), so the list is rewritten in place; order
+            // does not matter.  The stream that arrives last publishes the count and leaves the meta words ready.
+            const int need = nn + 1;
+            int base = 0;
+            if (lane == 0) base = atomicAdd(p.list_meta + kListAccum, need);
+            base = __shfl_sync(kFull, base, 0);
+            for (int j = lane; j < need; j += 32) p.next_list[base + j] = static_cast<int>(row0) + j;
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence();
+                if (atomicAdd(p.list_meta + kListArrived, 1) == p.B - 1) {
+                    __threadfence();
+                    p.list_meta[kListCount] = atomicExch(p.list_meta + kListAccum, 0);
+                    p.list_meta[kListSig] = row_list_sig(p.B, K);
+                    p.list_meta[kListArrived] = 0;
+                }
+            }
         }
     }
 }

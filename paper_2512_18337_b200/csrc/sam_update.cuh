@@ -66,8 +66,34 @@ struct UpdateArgs {
     int n_rec, n_seg, n_root, n_tail, root_span;
 };
 
+// Optional tail of the update kernel: once every block has finished scattering, the block that finishes last moves
+// the caller's stream states to the states that now hold their strings (what renormalize_kernel does), so that one
+// launch is all that stands between an update and the next decoding step.  B == 0: no tail.
+struct RenormTail {
+    DeviceSam sam;            // the view AFTER the update (state count included)
+    int B;
+    int* state;               // [B] in place
+    const int* matched_len;   // [B]
+    unsigned* blocks_done;    // zero between launches
+};
+
+// Climb suffix links until len(link(s)) < L <= len(s).  `fresh` = read past L1 and the read-only path: the records
+// may have been written moments ago by other blocks of the same kernel.
+template <bool fresh>
+__device__ __forceinline__ int renormalized_state(const DeviceSam& sam, int s, int L) {
+    if (s <= 0 || s >= sam.n_states || L < 0) return s;      // the walk kernels reset such pairs themselves
+    for (int hop = 0; hop < (1 << 30) && s != 0; ++hop) {
+        const int link = fresh ? __ldcg(&sam.rec[s].link) : __ldg(&sam.rec[s].link);
+        if (link < 0 || link >= sam.n_states) break;
+        const int link_len = (link == 0) ? 0 : (fresh ? __ldcg(&sam.rec[link].len) : __ldg(&sam.rec[link].len));
+        if (L > link_len) break;
+        s = link;
+    }
+    return s;
+}
+
 __global__ void __launch_bounds__(256)
-apply_update_kernel(UpdateArgs a) {
+apply_update_kernel(UpdateArgs a, RenormTail t) {
     const int nthreads = gridDim.x * blockDim.x;
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
@@ -91,31 +117,39 @@ apply_update_kernel(UpdateArgs a) {
     const int32_t* rtok = reinterpret_cast<const int32_t*>(a.stage + a.off_rtok);
     const int32_t* rdst = reinterpret_cast<const int32_t*>(a.stage + a.off_rdst);
     for (int i = gtid; i < a.n_root; i += nthreads) {
-        const int t = rtok[i];
-        if (t >= 0 && t < a.root_span) a.root[t] = rdst[i];
+        const int tk = rtok[i];
+        if (tk >= 0 && tk < a.root_span) a.root[tk] = rdst[i];
     }
     const int32_t* tail = reinterpret_cast<const int32_t*>(a.stage + a.off_tail);
     for (int i = gtid; i < a.n_tail; i += nthreads) a.corpus[i] = tail[i];
+
+    if (t.B > 0) {
+        __shared__ int is_last;
+        __threadfence();                      // this thread's writes before the block's arrival
+        __syncthreads();
+        if (threadIdx.x == 0) is_last = (atomicAdd(t.blocks_done, 1u) == gridDim.x - 1);
+        __syncthreads();
+        if (is_last) {
+            __threadfence();                  // every block has arrived: its writes are visible from here on
+            for (int b = threadIdx.x; b < t.B; b += blockDim.x) {
+                const int s0 = t.state[b];
+                const int s = renormalized_state<true>(t.sam, s0, t.matched_len[b]);
+                if (s != s0) t.state[b] = s;
+            }
+            if (threadIdx.x == 0) *t.blocks_done = 0u;
+        }
+    }
 }
 
 // After the text has grown, a stream's string of length L may belong to a state that was split off
-// its old one: the state of a string is the one with len(link(s)) < L <= len(s).  Climb suffix links
-// until that holds.  One thread per stream.
+// its old one: the state of a string is the one with len(link(s)) < L <= len(s) (renormalized_state).
+// One thread per stream.
 __global__ void __launch_bounds__(128)
 renormalize_kernel(DeviceSam sam, int B, int* __restrict__ state, const int* __restrict__ matched_len) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    int s = state[b];
-    const int L = matched_len[b];
-    if (s <= 0 || s >= sam.n_states || L < 0) return;      // the walk kernels reset such pairs themselves
-    const int s0 = s;
-    for (int hop = 0; hop < (1 << 30) && s != 0; ++hop) {
-        const int link = __ldg(&sam.rec[s].link);
-        if (link < 0 || link >= sam.n_states) break;
-        const int link_len = (link == 0) ? 0 : __ldg(&sam.rec[link].len);
-        if (L > link_len) break;
-        s = link;
-    }
+    const int s0 = state[b];
+    const int s = renormalized_state<false>(sam, s0, matched_len[b]);
     if (s != s0) state[b] = s;
 }
 
@@ -126,17 +160,8 @@ renormalize_slots_kernel(DeviceSam sam, int member, int n, const int* __restrict
                          const int* __restrict__ matched_len) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n || slots[i] != member) return;
-    int s = state[i];
-    const int L = matched_len[i];
-    if (s <= 0 || s >= sam.n_states || L < 0) return;
-    const int s0 = s;
-    for (int hop = 0; hop < (1 << 30) && s != 0; ++hop) {
-        const int link = __ldg(&sam.rec[s].link);
-        if (link < 0 || link >= sam.n_states) break;
-        const int link_len = (link == 0) ? 0 : __ldg(&sam.rec[link].len);
-        if (L > link_len) break;
-        s = link;
-    }
+    const int s0 = state[i];
+    const int s = renormalized_state<false>(sam, s0, matched_len[i]);
     if (s != s0) state[i] = s;
 }
 

@@ -76,11 +76,14 @@ def test_draft_parity_while_the_text_grows(seed, compact_every):
                                 rng.integers(sep + 1, sep + 50, size=5).astype(np.int32)]).astype(np.int32)
         osam.extend(piece)
         S.sam_extend(index.handle, piece)
-        assert S.sam_sync(index.handle) == osam.n
         before = st_o.copy()
         osam.renormalize(st_o, ml_o)
         moved += int((before != st_o).sum())
-        S.sam_renormalize(index.handle, B, st, ml)
+        if rnd % 2 == 0:
+            assert S.sam_sync(index.handle) == osam.n
+            S.sam_renormalize(index.handle, B, st, ml)
+        else:                                   # the same in one call (one kernel when the update is small)
+            assert S.sam_sync_renormalize(index.handle, B, st, ml) == osam.n
         torch.cuda.synchronize()
         assert (st.cpu().numpy() == st_o).all()
         # n_new = 0: the draft is re-emitted from the (moved) state over the grown text
@@ -135,8 +138,7 @@ def test_closed_loop_with_committed_tokens_appended():
             cpu.sam.extend(piece)
             cpu.sam.renormalize(cpu.state, cpu.mlen)
             S.sam_extend(index.handle, piece)
-            S.sam_sync(index.handle)
-            S.sam_renormalize(index.handle, cfg.B, gpu.state, gpu.mlen)
+            S.sam_sync_renormalize(index.handle, cfg.B, gpu.state, gpu.mlen)
             # the pending drafts came from the text before it grew; both sides re-emit them
             z = np.zeros((cfg.B, 1), np.int32)
             nz = np.zeros(cfg.B, np.int32)
@@ -201,7 +203,11 @@ def test_small_and_large_updates_take_their_own_paths():
         osam.extend(piece)
         inc0, full0, bytes0 = S.sam_update_stats(index.handle)
         S.sam_extend(index.handle, piece)
-        assert S.sam_sync(index.handle) == osam.n
+        if rnd < 3:
+            assert S.sam_sync(index.handle) == osam.n
+            S.sam_renormalize(index.handle, B, st, ml)
+        else:                                   # one call; after a large update the states get a kernel of their own
+            assert S.sam_sync_renormalize(index.handle, B, st, ml) == osam.n
         inc1, full1, bytes1 = S.sam_update_stats(index.handle)
         assert inc1 + full1 > inc0 + full0
         if n >= 25000:
@@ -209,7 +215,6 @@ def test_small_and_large_updates_take_their_own_paths():
         elif full1 == full0:
             assert bytes1 - bytes0 < (1 << 20)
         osam.renormalize(st_o, ml_o)
-        S.sam_renormalize(index.handle, B, st, ml)
         toks = np.empty((B, ld), np.int32)
         for b in range(B):
             start = int(rng.integers(0, osam.n - ld))

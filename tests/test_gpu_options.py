@@ -61,10 +61,14 @@ def test_verify_skipping_unused_rows(V, pad, B, K, variant):
     assert S.sam_workspace_status(ws, B, K) == 0
 
 
-@pytest.mark.parametrize("variant,skip", [(0, True), (0, False), (1, True), (2, False), (3, True), (3, False)])
+@pytest.mark.parametrize("variant,skip", [(0, True), (0, False), (1, True), (2, False), (3, True), (3, False),
+                                          (0, "chain"), (1, "chain"), (3, "chain")])
 def test_closed_loop_with_the_adaptive_switch(variant, skip):
     """A schedule of context lengths drives the switch: steps over the threshold run without speculation.
-    Every output of every step and the final counters equal the oracle's."""
+    Every output of every step and the final counters equal the oracle's.  skip = "chain": rows beyond the
+    proposal are skipped and, from the second step on, the rows to read come from the list the previous step's
+    accept kernel left in the workspace (SAM_STEP_ROW_LIST_READY) instead of a listing kernel."""
+    chain, skip = skip == "chain", bool(skip)
     cfg = W.CONFIGS[1].scaled(sessions=24, B=40, steps=14, vocab=20000)
     corpus = W.make_corpus(cfg)
     scripts = W.make_scripts(cfg, corpus)
@@ -86,6 +90,10 @@ def test_closed_loop_with_the_adaptive_switch(variant, skip):
             on = S.sam_adaptive_switch(ctx_schedule[t], cfg.B, 32768, 64)
             assert on == oracle.speculation_enabled(ctx_schedule[t], cfg.B, 32768, 64)
             flags = (0 if on else S.SAM_STEP_NO_SPECULATION) | (S.SAM_STEP_SKIP_UNUSED_ROWS if skip else 0)
+            oracle_flags = flags
+            if chain and t > 0:
+                flags |= S.SAM_STEP_ROW_LIST_READY
+            launches0 = S.sam_launch_count()
             off_steps += not on
             zero = np.zeros(cfg.B, np.int32)
             ow_g = f_g.overwrites(t, dg, ndg if on else zero)
@@ -101,7 +109,9 @@ def test_closed_loop_with_the_adaptive_switch(variant, skip):
             g = dict(argmax=gpu.argmax.cpu().numpy(), accepted=gpu.accepted.cpu().numpy(),
                      n_accepted=gpu.n_accepted.cpu().numpy(), drafts=gpu.drafts.cpu().numpy(),
                      n_draft=gpu.n_draft.cpu().numpy(), state=gpu.state.cpu().numpy(), matched_len=gpu.mlen.cpu().numpy())
-            o = cpu.sam.step_ex(cpu.bits, c.B, c.K, c.vocab, do, ndo, cpu.state, cpu.mlen, c.min_match, flags, cnt_o)
+            if chain and t > 0 and on:
+                assert S.sam_launch_count() - launches0 == 2       # argmax + accept, no listing kernel
+            o = cpu.sam.step_ex(cpu.bits, c.B, c.K, c.vocab, do, ndo, cpu.state, cpu.mlen, c.min_match, oracle_flags, cnt_o)
             o["state"], o["matched_len"] = cpu.state.copy(), cpu.mlen.copy()
             gpu.unpoke(ow_g["row"], ow_g["col"], sv_g)
             cpu.unpoke(ow_o["row"], ow_o["col"], sv_o)
@@ -118,9 +128,117 @@ def test_closed_loop_with_the_adaptive_switch(variant, skip):
     assert gpu.status() == 0
 
 
+def test_closed_loop_driven_by_the_counter_switch():
+    """The switch decided from the device counters: after every window of two steps the counters of the window's
+    speculating passes go to sam_speculation_pays together with the cost ratio of the moment (a schedule standing
+    in for a load that changes: cheap verification, then a phase where a full pass costs 40 one-row passes, then
+    cheap again).  While speculation is off every third window tries it again.  The library's decisions equal the
+    oracle's, every output of every step equals the oracle's, and the switch goes off and comes back on."""
+    cfg = W.CONFIGS[1].scaled(sessions=24, B=40, steps=24, vocab=20000)
+    corpus = W.make_corpus(cfg)
+    scripts = W.make_scripts(cfg, corpus)
+    noise = W.make_noise_logits(cfg)
+    rowmax = W.f32_to_bf16_bits(W.bf16_bits_to_f32(noise).max(axis=1))
+    gpu = CudaBackend(cfg, corpus, bits_to_device(noise))
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    f_g, f_o = W.ClosedLoopFeeder(cfg, scripts, rowmax), W.ClosedLoopFeeder(cfg, scripts, rowmax)
+    toks, n = f_g.prime_tokens()
+    dg, ndg = gpu.prime(toks, n)
+    do, ndo = cpu.prime(toks, n)
+    cnt_g = torch.zeros(S.SAM_N_COUNTERS, dtype=torch.int64, device=DEV)
+    cnt_o = np.zeros(6, np.int64)
+    ratio_of_window = [1.2, 1.2, 1.2, 40.0, 40.0, 40.0, 40.0, 40.0, 1.2, 1.2, 1.2, 1.2]
+    on, windows_off, history = True, 0, []
+    c = cfg
+    for t in range(cfg.steps):
+        w = t // 2
+        flags = S.SAM_STEP_SKIP_UNUSED_ROWS | (0 if on else S.SAM_STEP_NO_SPECULATION)
+        zero = np.zeros(cfg.B, np.int32)
+        ow_g = f_g.overwrites(t, dg, ndg if on else zero)
+        ow_o = f_o.overwrites(t, do, ndo if on else zero)
+        keep = np.arange(ow_g["row"].shape[0])
+        sv_g = gpu.poke(ow_g["row"], ow_g["col"], ow_g["bits"], keep)
+        sv_o = cpu.poke(ow_o["row"], ow_o["col"], ow_o["bits"], keep)
+        S.sam_step_ex(gpu.index.handle, gpu.logits, gpu.stride, c.B, c.K, c.vocab, gpu.drafts, gpu.n_draft,
+                      gpu.argmax, gpu.accepted, gpu.n_accepted, gpu.state, gpu.mlen, c.min_match,
+                      gpu.drafts, gpu.n_draft, flags, cnt_g, gpu.ws, gpu.ws_bytes)
+        torch.cuda.synchronize()
+        g = dict(argmax=gpu.argmax.cpu().numpy(), accepted=gpu.accepted.cpu().numpy(),
+                 n_accepted=gpu.n_accepted.cpu().numpy(), drafts=gpu.drafts.cpu().numpy(),
+                 n_draft=gpu.n_draft.cpu().numpy(), state=gpu.state.cpu().numpy(), matched_len=gpu.mlen.cpu().numpy())
+        o = cpu.sam.step_ex(cpu.bits, c.B, c.K, c.vocab, do, ndo, cpu.state, cpu.mlen, c.min_match, flags, cnt_o)
+        o["state"], o["matched_len"] = cpu.state.copy(), cpu.mlen.copy()
+        gpu.unpoke(ow_g["row"], ow_g["col"], sv_g)
+        cpu.unpoke(ow_o["row"], ow_o["col"], sv_o)
+        for k in KEYS:
+            assert (g[k] == o[k]).all(), (t, k)
+        f_g.advance(g["n_accepted"])
+        f_o.advance(o["n_accepted"])
+        dg, ndg, do, ndo = g["drafts"], g["n_draft"], o["drafts"], o["n_draft"]
+        if t % 2 == 1:                                    # end of a window
+            host = cnt_g.cpu().numpy()
+            assert (host == cnt_o).all()
+            if on:                                        # only speculating passes say what speculation is worth
+                on = S.sam_speculation_pays(host, c.K, ratio_of_window[w])
+                assert on == oracle.speculation_pays(cnt_o, c.K, ratio_of_window[w])
+                windows_off = 0
+            else:
+                windows_off += 1
+                on = windows_off % 3 == 0                 # try again every third window
+            history.append(on)
+            cnt_g.zero_()
+            cnt_o[:] = 0
+    assert gpu.status() == 0
+    # on through the cheap phase, off (with failed retries) through the expensive one, on again afterwards
+    assert history[:2] == [True, True] and not any(history[3:5]) and history[-1] and history.count(False) >= 4
+    k = history.index(False)
+    assert True in history[k:], history
+
+
+def test_row_list_ready_without_a_list_is_reported():
+    """SAM_STEP_ROW_LIST_READY on a workspace that holds no list for this shape: nothing is read, the status word
+    says so, and after re-initialising the workspace an ordinary call gives the oracle's result."""
+    cfg = W.CONFIGS[0]
+    corpus = W.make_corpus(cfg)
+    noise = W.make_noise_logits(cfg)
+    gpu = CudaBackend(cfg, corpus, bits_to_device(noise))
+    cpu = OracleBackend(cfg, corpus, noise.copy())
+    toks = np.ascontiguousarray(W.make_scripts(cfg, corpus)[:, :cfg.prime])
+    n = np.full(cfg.B, cfg.prime, np.int32)
+    gpu.prime(toks, n)
+    do, ndo = cpu.prime(toks, n)
+    st0, ml0, d0, nd0 = (x.clone() for x in (gpu.state, gpu.mlen, gpu.drafts, gpu.n_draft))
+    both = S.SAM_STEP_SKIP_UNUSED_ROWS | S.SAM_STEP_ROW_LIST_READY
+    for variant in (1, 3):
+        S.sam_set_argmax_variant(variant)
+        try:
+            S.sam_workspace_init(gpu.ws, gpu.ws_bytes)        # whatever list an earlier call left is gone
+            gpu.flags = both
+            gpu.launch_step()
+            torch.cuda.synchronize()
+            assert gpu.status() == 3
+            S.sam_workspace_init(gpu.ws, gpu.ws_bytes)
+            for dst, src in ((gpu.state, st0), (gpu.mlen, ml0), (gpu.drafts, d0), (gpu.n_draft, nd0)):
+                dst.copy_(src)
+            gpu.flags = S.SAM_STEP_SKIP_UNUSED_ROWS
+            g = gpu.step(None, None)
+            assert gpu.status() == 0
+        finally:
+            S.sam_set_argmax_variant(0)
+        o = cpu.sam.step_ex(cpu.bits, cfg.B, cfg.K, cfg.vocab, do, ndo, cpu.state.copy(), cpu.mlen.copy(), cfg.min_match,
+                            S.SAM_STEP_SKIP_UNUSED_ROWS, np.zeros(6, np.int64))
+        for k in ("argmax", "accepted", "n_accepted", "drafts", "n_draft"):
+            assert (g[k] == o[k]).all(), (variant, k)
+        for dst, src in ((gpu.state, st0), (gpu.mlen, ml0), (gpu.drafts, d0), (gpu.n_draft, nd0)):
+            dst.copy_(src)
+
+
 def test_flags_are_checked():
     lib = S.binding._load()
     assert lib.sam_verify_ex(None, 8, 1, 1, 8, None, None, None, None, None, 4, None, None, 0, None) == -1
+    # the row-list flag belongs to sam_step_ex and needs the row-skipping flag beside it
+    assert lib.sam_step_ex(None, None, 8, 1, 1, 8, None, None, None, None, None, None, None, 1, None, None, 4, None,
+                           None, 0, None) == -1
     assert lib.sam_adaptive_switch(10, 10, 10, 10) == 1 and lib.sam_adaptive_switch(11, 10, 10, 10) == 0
 
 
