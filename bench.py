@@ -39,16 +39,17 @@ import workload as W  # noqa: E402
 METRIC = "sam_draft_verify_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one argmax launch, per logits row, from the ncu
-# capture summarised in profiles/launch_list_cfg2.md (config 2, argmax_bulk_kernel; traffic scales with rows)
-NCU_DRAM_BYTES_PER_ROW = 304325.1
-# the same for argmax_direct_kernel (--variant 1; profiles/argmax_direct_kernel_cfg2_launch_list.md); that capture was
-# taken at V = 151,936, and the figure is only reported for that row length
-NCU_DRAM_BYTES_PER_ROW_DIRECT = 304694.3
-# and for the same kernel on the paper's evaluation shape (config 5: 16 rows per launch; used for workloads that fit in L2)
-NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE = 305051.8
-# dram__sectors_read.sum of one accept_kernel launch per stream, same workload (profiles/walk_kernels_cfg2_sectors.md)
-NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 46.9
+# DRAM traffic of one argmax_bulk_kernel launch from the ncu captures summarised in
+# profiles/argmax_bulk_kernel_cfg1_ncu_full.md (config 1, four launches of the kernel as it stands): dram__bytes_read.sum per
+# logits row (every row is read once, so the reads grow in proportion to the rows) and dram__bytes_write.sum per launch
+# (write-backs of the harness' sparse planting, which do not grow with the rows; the kernel writes 8 bytes per row)
+NCU_DRAM_READ_BYTES_PER_ROW = 304105.3
+NCU_DRAM_WRITE_BYTES_PER_LAUNCH = 2.82e6
+# the same for argmax_direct_kernel (profiles/argmax_direct_kernel_cfg1_dram.md), captured at V = 151,936 and only
+# reported for that row length
+NCU_DRAM_READ_BYTES_PER_ROW_DIRECT = None
+# dram__sectors_read.sum of one accept_kernel launch per stream, config 2 (profiles/walk_kernels_cfg2_sectors.md)
+NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 45.8
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -509,9 +510,7 @@ def run_ours(args):
     direct = args.variant == 1 or (args.variant == 0 and cfg.K <= 16 and R * cfg.vocab * 2 <= (768 << 20))
     traffic_per_row = None
     if cfg.vocab == 151936:
-        traffic_per_row = (NCU_DRAM_BYTES_PER_ROW if not direct else
-                           NCU_DRAM_BYTES_PER_ROW_DIRECT if R * cfg.vocab * 2 > (126 << 20) else
-                           NCU_DRAM_BYTES_PER_ROW_LATENCY_CASE)
+        traffic_per_row = NCU_DRAM_READ_BYTES_PER_ROW_DIRECT if direct else NCU_DRAM_READ_BYTES_PER_ROW
     achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
     walk = None
     if split is not None:
@@ -537,7 +536,8 @@ def run_ours(args):
         "launches_per_step": launches_per_step, "variant": args.variant, "cuda_graph": bool(args.graph), "back_to_back": back_to_back,
         "roofline": {"kernel": kernel_name + (" (argmax_direct_kernel)" if direct else " (argmax_bulk_kernel)" if launches_per_step != 1 else ""), "kernel_ms": kernel_ms, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0,
-                     "traffic": traffic_per_row * (rows_read_per_step if args.skip_unused_rows else R) if traffic_per_row else None,
+                     "traffic": (traffic_per_row * (rows_read_per_step if args.skip_unused_rows else R)
+                                 + NCU_DRAM_WRITE_BYTES_PER_LAUNCH) if traffic_per_row else None,
                      "algorithmic_bytes": alg_bytes,
                      "whole_step": {"ms": total_ms / args.steps, "achieved": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9,
                                     "frac": alg_bytes / (total_ms / args.steps * 1e-3) / 1e9 / peak,

@@ -388,9 +388,10 @@ enum : int { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusQueueOverflow = 2, kS
 //                  the list counts only if meta[kListSig] == sig (it was made for this batch shape), otherwise
 //                  nothing is reduced and *status is raised.  list == nullptr: all rows 0..R-1.
 //   v_offset:      added to every index (the logits are columns v_offset.. of a wider vocabulary).
-// meta words: [kListCount] rows in the list; [kListAccum] rows collected so far for the NEXT list (zero between
-// calls); [kListArrived] streams that have added theirs (zero between calls); [kListSig] shape the list was made for.
-enum : int { kListCount = 0, kListAccum = 1, kListArrived = 2, kListSig = 3 };
+// meta words: [kListCount] rows in the list; [kListSig] the shape the list was made for; [kListAccum], 8-byte aligned,
+// a 64-bit word zero between calls: rows collected so far for the NEXT list (low half) and streams that have added
+// theirs (high half).
+enum : int { kListCount = 0, kListSig = 1, kListAccum = 2 };
 struct RowMap {
     const int* list;
     const int* meta;
@@ -700,21 +701,20 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         if (p.next_list != nullptr) {
             // The rows the next step will need from this stream go into the next row list.  The argmax kernel that
             // read the current list has finished (this kernel waited for it), so the list is rewritten in place; order
-            // does not matter.  The stream that arrives last publishes the count and leaves the meta words ready.
+            // does not matter.  One 64-bit atomic per stream both reserves the stream's places and counts the streams
+            // that have come by; the last one publishes the total and leaves the word zero for the next step.  The
+            // reader is the next kernel in the stream, so no ordering is needed between a stream's entries and the total.
             const int need = nn + 1;
-            int base = 0;
-            if (lane == 0) base = atomicAdd(p.list_meta + kListAccum, need);
-            base = __shfl_sync(kFull, base, 0);
+            unsigned long long old = 0ull;
+            unsigned long long* accum = reinterpret_cast<unsigned long long*>(p.list_meta + kListAccum);
+            if (lane == 0) old = atomicAdd(accum, (1ull << 32) | static_cast<unsigned long long>(need));
+            old = __shfl_sync(kFull, old, 0);
+            const int base = static_cast<int>(old & 0xFFFFFFFFull);
             for (int j = lane; j < need; j += 32) p.next_list[base + j] = static_cast<int>(row0) + j;
-            __syncwarp();
-            if (lane == 0) {
-                __threadfence();
-                if (atomicAdd(p.list_meta + kListArrived, 1) == p.B - 1) {
-                    __threadfence();
-                    p.list_meta[kListCount] = atomicExch(p.list_meta + kListAccum, 0);
-                    p.list_meta[kListSig] = row_list_sig(p.B, K);
-                    p.list_meta[kListArrived] = 0;
-                }
+            if (lane == 0 && static_cast<int>(old >> 32) == p.B - 1) {
+                p.list_meta[kListCount] = base + need;
+                p.list_meta[kListSig] = row_list_sig(p.B, K);
+                *accum = 0ull;
             }
         }
     }

@@ -183,6 +183,58 @@ def test_builder_thread_and_empty_start():
     assert (ml_o == ld).all()
 
 
+def test_updates_pile_up_and_ring_slots_are_reused():
+    """The builder thread sends every small update to one of eight slots of the device blob ahead of time.  Twenty
+    updates between two syncs overflow the ring: the first eight wait in their slots, the others travel on the
+    caller's stream when sam_sync comes, all applied in order.  Then many rounds of a few updates each make every
+    slot be used again and again.  After every sync the device copy drafts like the oracle's automaton."""
+    rng = np.random.default_rng(23)
+    sep, K, mm, B, ld = 1000, 6, 2, 48, 10
+    text = _hub_text(rng, 1500, sep)
+    index = S.SamIndex(text, [sep], max_tokens=60000, max_token_id=sep + 50)
+    osam = oracle.OracleSAM(text, [sep])
+    st = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ml = torch.zeros(B, dtype=torch.int32, device=DEV)
+    st_o = np.zeros(B, np.int32)
+    ml_o = np.zeros(B, np.int32)
+    bursts = [20] + [3, 1, 5, 2] * 6
+    for rnd, n_updates in enumerate(bursts):
+        inc0, full0, _ = S.sam_update_stats(index.handle)
+        for _ in range(n_updates):
+            piece = np.concatenate([[sep], _hub_text(rng, int(rng.integers(5, 120)), sep)]).astype(np.int32)
+            osam.extend(piece)
+            S.sam_extend(index.handle, piece)              # waits for the builder thread: one update per piece
+        osam.renormalize(st_o, ml_o)
+        if rnd % 2 == 0:
+            assert S.sam_sync_renormalize(index.handle, B, st, ml) == osam.n
+        else:
+            assert S.sam_sync(index.handle) == osam.n
+            S.sam_renormalize(index.handle, B, st, ml)
+        inc1, full1, _ = S.sam_update_stats(index.handle)
+        assert (inc1 - inc0) + (full1 - full0) == n_updates
+        toks = np.empty((B, ld), np.int32)
+        for b in range(B):
+            start = int(rng.integers(0, osam.n - ld))
+            toks[b] = osam.corpus[start:start + ld]
+        toks[rng.random((B, ld)) < 0.05] = sep + 9
+        n_new = rng.integers(0, ld + 1, size=B).astype(np.int32)
+        _draft_both(index, osam, B, st, ml, st_o, ml_o, toks, n_new, K, mm)
+    ex, oe = S.sam_export(index.handle), osam.export()
+    for k in oe:
+        assert (ex[k] == oe[k]).all(), k
+
+
+def test_sync_without_pending_updates_launches_nothing():
+    rng = np.random.default_rng(4)
+    sep = 500
+    index = S.SamIndex(_hub_text(rng, 800, sep), [sep], max_tokens=4000, max_token_id=sep)
+    st = torch.zeros(8, dtype=torch.int32, device=DEV)
+    ml = torch.zeros(8, dtype=torch.int32, device=DEV)
+    n0 = S.sam_launch_count()
+    assert S.sam_sync_renormalize(index.handle, 8, st, ml) == 800
+    assert S.sam_launch_count() == n0
+
+
 def test_small_and_large_updates_take_their_own_paths():
     """Updates of a few hundred tokens go through one page-locked buffer, one copy and one kernel; an update of
     tens of thousands of tokens is too large for that buffer and is applied section by section.  Both leave the
