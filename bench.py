@@ -40,14 +40,15 @@ METRIC = "sam_draft_verify_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one argmax_bulk_kernel launch from the ncu captures summarised in
-# profiles/argmax_bulk_kernel_cfg1_ncu_full.md (config 1, four launches of the kernel as it stands): dram__bytes_read.sum per
+# profiles/argmax_bulk_kernel_cfg1_ncu_full.md and profiles/argmax_direct_kernel_cfg1_dram.md (config 1, launches of the
+# kernel as it stands): dram__bytes_read.sum per
 # logits row (every row is read once, so the reads grow in proportion to the rows) and dram__bytes_write.sum per launch
 # (write-backs of the harness' sparse planting, which do not grow with the rows; the kernel writes 8 bytes per row)
 NCU_DRAM_READ_BYTES_PER_ROW = 304105.3
 NCU_DRAM_WRITE_BYTES_PER_LAUNCH = 2.82e6
 # the same for argmax_direct_kernel (profiles/argmax_direct_kernel_cfg1_dram.md), captured at V = 151,936 and only
 # reported for that row length
-NCU_DRAM_READ_BYTES_PER_ROW_DIRECT = None
+NCU_DRAM_READ_BYTES_PER_ROW_DIRECT = 304549.0
 # dram__sectors_read.sum of one accept_kernel launch per stream, config 2 (profiles/walk_kernels_cfg2_sectors.md)
 NCU_ACCEPT_DRAM_SECTORS_PER_STREAM = 45.8
 

@@ -99,11 +99,13 @@ void sam_free(sam_index* idx);
 
 /* Bytes of device scratch sam_verify / sam_step need for B streams and draft length K
  * (one 64-bit partial result per logits row, the walk-ahead states of every draft position, one
- * completion counter per stream, a row list and a status word).  Returns a negative SAM_ERR_* on bad sizes. */
+ * completion counter per stream and per row, a row list with its bookkeeping words and a status word).
+ * Returns a negative SAM_ERR_* on bad sizes. */
 int64_t sam_workspace_bytes(int32_t B, int32_t K);
 
 /* Zero-fills the scratch (device, 8-byte aligned) on the stream.  Required once before the
- * first sam_verify / sam_step that uses it; every successful call leaves it ready for the next one.
+ * first sam_verify / sam_step that uses it; every successful call leaves it ready for the next one
+ * (not all zero: a row list for the next step and a count of launches may stay in it).
  * Call it again after a hot-path call returned an error.  Calls that share one workspace
  * must not overlap on the device. */
 int sam_workspace_init(void* workspace, int64_t bytes, void* cuda_stream);
@@ -472,8 +474,10 @@ int sam_profile_enable(int32_t max_calls);
  *       the direct-load kernel otherwise; each followed by the accept kernel as a dependent launch;
  *   1 = always the direct-load kernel;
  *   2 = the bulk-copy kernel whenever the rows are aligned, with the accept step of every stream
- *       inside it, run as soon as the stream's rows are complete (one launch per call; measured
- *       slightly slower than two launches on B200);
+ *       inside it: every CTA takes the rows its streams' proposals use (0 .. n_draft) first, a stream's
+ *       accept step runs as soon as those rows are complete, and the rows behind the proposals are
+ *       reported by the kernel when they are (one launch per call; measured slower than two launches
+ *       on B200, so not the default; rows too short for 48 KB tiles fall back to two launches);
  *   3 = the bulk-copy kernel whenever the rows are aligned, followed by the accept kernel. */
 int sam_set_argmax_variant(int32_t variant);
 int32_t sam_profile_count(void);

@@ -24,11 +24,15 @@
 //
 // Fused tail.  When the host asks for it, the accept step of a stream (decode the row results,
 // longest matching prefix, follow the model's own token, next draft) runs inside this kernel as
-// soon as the last partial result of the stream's K+1 rows has landed: after publishing a row the
-// finisher adds the tiles this CTA reduced for it to a per-stream counter, the addition that
-// completes the count puts the stream into a queue in the CTA's shared memory, and idle warps of
+// soon as the rows it needs are complete.  It needs rows 0 .. n_draft[b] only (the rows behind the proposal
+// are reported, nothing depends on them), so every CTA takes the used rows of its share first and the
+// others afterwards: the accept steps then run under the second half of the stream instead of after it.
+// A finished row is complete at once when the CTA had all its tiles; a row shared with the neighbouring
+// CTA is complete when a counter says so.  A complete used row adds one to its stream's counter, the
+// addition that completes the stream puts it into a queue in the CTA's shared memory, and idle warps of
 // that CTA (the walk-ahead warps, the finisher and the consumer warps once their work is done) take
-// streams from the queue.  Nobody waits for another CTA, so the scheme needs no co-residency.
+// streams from the queue; a complete row behind the proposal is decoded into argmax_out by the finisher
+// itself.  Nobody waits for another CTA, so the scheme needs no co-residency.
 //
 // Every wait on an mbarrier is bounded: after kMaxPolls unsuccessful polls the waiting thread
 // raises the CTA's abort flag and the status word in global memory, all roles leave their
@@ -99,7 +103,9 @@ constexpr int kQueueCap = 1024;                        // streams one CTA can be
 constexpr size_t kBulkCtrlOff = static_cast<size_t>(kBulkRingBytes);
 constexpr size_t kBulkQueueOff = kBulkCtrlOff + 1024;
 constexpr size_t kBulkCandOff = kBulkQueueOff + kQueueCap * 4;
-constexpr size_t kBulkSmemBytes = kBulkCandOff + static_cast<size_t>(kRowSlots) * kBulkConsumerWarps * 8;
+constexpr int kOrderCap = 1024;                        // rows of a CTA that can be taken in another order than they lie
+constexpr size_t kBulkOrderOff = kBulkCandOff + static_cast<size_t>(kRowSlots) * kBulkConsumerWarps * 8;
+constexpr size_t kBulkSmemBytes = kBulkOrderOff + static_cast<size_t>(kOrderCap) * 4;
 
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -166,28 +172,46 @@ struct BulkShared {
 };
 static_assert(sizeof(BulkShared) <= 1024, "control block");
 
-// Fused accept step (see the file header).  `done[b]` counts contributions to stream b and is
-// zero between calls; `expected` is the count at which the stream is complete.
+// Fused accept step (see the file header).  `done[b]` counts the contributions to stream b that have arrived and
+// `rowcnt[r]` the tiles of a shared row; both are zero between calls.
 struct FusedTail {
     AcceptArgs args;
-    int* done;       // [B]
-    int expected;
+    int* done;       // [B] contributions that have arrived: the stream's used rows (0..n_draft), + 1 for its walk-ahead
+    int* rowcnt;     // [R] tiles reduced so far of a row that two CTAs share
+    int prewalk;     // 1: the walk-ahead of a stream counts as one of its contributions
     int mode;        // 0 = off, else kTailVerifyOnly + 1 or kTailResume + 1
+    int* launch_words;   // [0] launches through this scratch so far, [1] CTAs of the current launch that have left
 };
+// Rows 0 .. n_draft[b] of stream b are the ones its accept step needs ("used"); returns their number.  n_draft is read
+// past the read-only path: the accept step of the stream may overwrite it in this very launch (next_n_draft may be the
+// same array).
+__device__ __forceinline__ int used_rows_of(const AcceptArgs& a, int b) {
+    return ((a.flags & kNoSpeculation) ? 0 : max(0, min(__ldcg(a.n_draft + b), a.K))) + 1;
+}
+// The same for a row that completes at an unknown time: once the stream's accept step has run in this launch, n_draft[b]
+// may already hold the NEXT proposal's length, and whatever completes after that step is a row behind the proposal
+// (the step waited for all the others).  The step writes the launch's number into acc_epoch[b], then a fence, then
+// n_draft; here the order is n_draft, fence, acc_epoch - so a count taken from n_draft is the old one whenever the
+// launch's number is not seen yet.
+__device__ __forceinline__ int used_rows_now(const FusedTail& ft, int epoch, int b) {
+    const int u = used_rows_of(ft.args, b);
+    __threadfence();
+    return (__ldcg(ft.args.acc_epoch + b) == epoch) ? 0 : u;
+}
 
 __device__ __forceinline__ int ld_volatile_s32(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
 __device__ __forceinline__ void st_volatile_s32(int* p, int v) { *reinterpret_cast<volatile int*>(p) = v; }
 
-__device__ __forceinline__ void fused_accept(const DeviceSam& sam, const FusedTail& ft, int b, int lane) {
+__device__ __forceinline__ void fused_accept(const DeviceSam& sam, const FusedTail& ft, int epoch, int b, int lane) {
     __threadfence();                 // order the reads below after the counter observation
-    if (ft.mode == kTailResume + 1) accept_stream<kTailResume>(sam, ft.args, b, lane);
-    else accept_stream<kTailVerifyOnly>(sam, ft.args, b, lane);
+    if (ft.mode == kTailResume + 1) accept_stream<kTailResume>(sam, ft.args, b, lane, nullptr, nullptr, epoch);
+    else accept_stream<kTailVerifyOnly>(sam, ft.args, b, lane, nullptr, nullptr, epoch);
     if (lane == 0) ft.done[b] = 0;
 }
 
 // Idle warps serve the CTA's queue until the finisher has left its loop and the queue is drained.
 // Each round takes one ticket; a ticket beyond the final tail means there is no more work.
-__device__ __forceinline__ void serve_queue(const DeviceSam& sam, const FusedTail& ft, BulkShared* sh,
+__device__ __forceinline__ void serve_queue(const DeviceSam& sam, const FusedTail& ft, int epoch, BulkShared* sh,
                                             const int* queue, volatile int* abort, int* status, int lane) {
     for (;;) {
         int b = -1;
@@ -213,7 +237,7 @@ __device__ __forceinline__ void serve_queue(const DeviceSam& sam, const FusedTai
         }
         b = __shfl_sync(kFull, b, 0);
         if (b < 0) return;
-        fused_accept(sam, ft, b, lane);
+        fused_accept(sam, ft, epoch, b, lane);
     }
 }
 
@@ -230,6 +254,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
     BulkShared* sh = reinterpret_cast<BulkShared*>(smem_raw + kBulkCtrlOff);
     int* queue = reinterpret_cast<int*>(smem_raw + kBulkQueueOff);
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem_raw + kBulkCandOff);   // [kRowSlots][warps]
+    int* order = reinterpret_cast<int*>(smem_raw + kBulkOrderOff);             // [kOrderCap] the CTA's rows in the order it takes them
 
     // the accept kernel may be scheduled now; it waits for this grid before it reads any result
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -262,8 +287,51 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
     }
     if (ft.mode != 0)
         for (int i = threadIdx.x; i < kQueueCap; i += blockDim.x) queue[i] = -1;
+    // With the accept step inside the kernel: the used rows (0 .. n_draft) of the CTA's share first, the rows behind the
+    // proposals afterwards.  One lane per stream of the share counts the stream's used and other rows inside the share,
+    // a warp-wide running sum gives every stream its two places, and the lane writes its stream's rows there.
+    // the number of this launch: one more than the launches that have gone through the scratch (a replayed graph counts too)
+    const int epoch = (ft.mode != 0) ? __ldcg(ft.launch_words) + 1 : 0;
+    const int K1 = ft.args.K + 1;
+    const long long b_first = (ft.mode != 0) ? row_first / K1 : 0;
+    const int n_streams = (ft.mode != 0 && n_rows > 0) ? static_cast<int>((row_first + n_rows - 1) / K1 - b_first + 1) : 0;
+    const bool ordered = ft.mode != 0 && plan.n_groups == 1 && n_rows > 0 && n_rows <= kOrderCap && n_streams <= 32;
+    if (ordered && warp == 0) {
+        int used = 0, rest = 0, j_lo = 0, j_hi = 0, u = 0;
+        if (lane < n_streams) {
+            const long long b = b_first + lane;
+            j_lo = static_cast<int>(max(0ll, row_first - b * K1));
+            j_hi = static_cast<int>(min(static_cast<long long>(K1), row_first + n_rows - b * K1));      // exclusive
+            u = used_rows_now(ft, epoch, static_cast<int>(b));
+            used = max(0, min(u, j_hi) - j_lo);
+            rest = (j_hi - j_lo) - used;
+        }
+        int used_before = used, rest_before = rest;                // inclusive running sums over the lanes
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int a = __shfl_up_sync(kFull, used_before, d), c = __shfl_up_sync(kFull, rest_before, d);
+            if (lane >= d) { used_before += a; rest_before += c; }
+        }
+        const int all_used = __shfl_sync(kFull, used_before, 31);
+        used_before -= used;
+        rest_before -= rest;
+        if (lane < n_streams) {
+            const int base = static_cast<int>((b_first + lane) * K1 - row_first);     // the stream's row 0 as a row of the share
+            for (int j = j_lo; j < j_hi; ++j) {
+                const int at = (j < u) ? used_before + (j - j_lo) : all_used + rest_before + (j - max(j_lo, u));
+                order[at] = base + j;
+            }
+        }
+    }
     __syncthreads();
     volatile int* abort = &sh->abort;
+    // The i-th row this CTA takes (as a position: in the list, or the row itself), and which of its tiles are the CTA's.
+    auto seq_row = [&](int i) -> long long { return row_first + (ordered ? order[i] : i); };
+    auto tiles_of = [&](long long r, int& lo, int& hi) {
+        const long long first = r * tiles_per_row;
+        lo = (t0 > first) ? static_cast<int>(t0 - first) : 0;
+        hi = (t1 - first < tiles_per_row) ? static_cast<int>(t1 - first) : tiles_per_row;
+    };
     // a row named by a list is clamped into the logits: a stale or foreign list can give wrong results, never a fault
     auto actual_row = [&](long long pos) -> long long {
         if (rm.list == nullptr) return pos;
@@ -276,27 +344,25 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         if (lane == 0) {
             long long it = 0;
             bool ok = true;
-            long long row = row_first;
-            int tile = static_cast<int>(t0 - row * tiles_per_row);
             int s = 0;
             uint32_t use = 0;
             const uint64_t policy = l2_evict_first_policy();
-            for (long long t = t0; t < t1; ++t, ++it) {
+            for (int i = 0; i < n_rows && ok; ++i) {
+                const long long row = seq_row(i);
+                int tile, tile_hi;
+                tiles_of(row, tile, tile_hi);
                 // with a row list the row number is fetched before the wait, off the path of the copy
-                const long long arow = actual_row(row);
-                if (!mbar_wait_bounded(&sh->empty[s], (use & 1u) ^ 1u, abort)) { ok = false; break; }
-                const int v0 = tile * tile_vec;
-                const int nv = max(0, min(tile_vec, nvec_row - v0));
-                if (nv > 0) {
+                const __nv_bfloat16* src = logits + actual_row(row) * stride;
+                for (; tile < tile_hi; ++tile, ++it) {
+                    if (!mbar_wait_bounded(&sh->empty[s], (use & 1u) ^ 1u, abort)) { ok = false; break; }
+                    const int v0 = tile * tile_vec;
+                    const int nv = max(0, min(tile_vec, nvec_row - v0));
                     const uint32_t bytes = static_cast<uint32_t>(nv) * 16u;
                     mbar_arrive_expect_tx(&sh->full[s], bytes);
                     bulk_load(stage_base + static_cast<size_t>(s) * plan.stage_bytes,
-                              reinterpret_cast<const uint4*>(logits + arow * stride) + v0, bytes, &sh->full[s], policy);
-                } else {
-                    mbar_arrive(&sh->full[s]);      // nothing to copy (row shorter than one vector)
+                              reinterpret_cast<const uint4*>(src) + v0, bytes, &sh->full[s], policy);
+                    if (++s == ns) { s = 0; ++use; }
                 }
-                if (++tile == tiles_per_row) { tile = 0; ++row; }
-                if (++s == ns) { s = 0; ++use; }
             }
             sh->issued = it;
             if (!ok) {
@@ -306,7 +372,6 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         }
     } else if (warp == kBulkConsumerWarps + 1) {
         // ------------------------------------------------------------------ finisher
-        const int K1 = ft.args.K + 1;
         int done_rows = 0;
         uint32_t polls = 0;
         while (done_rows < n_rows) {
@@ -330,7 +395,8 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             const int n = min(32, p - done_rows);
             if (lane < n) {
                 const int i = done_rows + lane;
-                const long long row = actual_row(row_first + i);
+                const long long pos = (plan.n_groups == 1) ? seq_row(i) : row_first + i;
+                const long long row = actual_row(pos);
                 const unsigned long long* c = cand + static_cast<size_t>(i % kRowSlots) * kBulkConsumerWarps;
                 unsigned long long k = 0ull;
 #pragma unroll
@@ -338,17 +404,43 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                     const unsigned long long x = (w < n_cons) ? c[w] : 0ull;
                     k = (x > k) ? x : k;
                 }
-                if (k != 0ull) atomicMax(keys + row, k);
-                if (ft.mode != 0) {
-                    __threadfence();                   // the candidate first, then the count
-                    const long long ra = row * tiles_per_row, rb = ra + tiles_per_row;
-                    const int seg = static_cast<int>(min(rb, t1) - max(ra, t0));   // tiles of the row this CTA reduced
-                    const int b = static_cast<int>(row / K1);
-                    if (atomicAdd(ft.done + b, seg) + seg == ft.expected) {
+                if (ft.mode == 0) {
+                    if (k != 0ull) atomicMax(keys + row, k);
+                } else {
+                    int lo, hi;
+                    tiles_of(pos, lo, hi);
+                    const int seg = hi - lo;           // tiles of the row this CTA reduced
+                    bool complete = seg == tiles_per_row;      // the row is this CTA's alone: k is its result
+                    if (!complete) {
+                        // shared with the neighbouring CTA: results meet in the row's word, a counter tells who came last
+                        if (k != 0ull) atomicMax(keys + row, k);
                         __threadfence();
-                        const int slot = atomicAdd(&sh->q_tail, 1);
-                        if (slot < kQueueCap) st_volatile_s32(queue + slot, b);
-                        else atomicExch(status, kStatusQueueOverflow);   // the host sizes the grid so that this cannot happen
+                        complete = atomicAdd(ft.rowcnt + row, seg) + seg == tiles_per_row;
+                        if (complete) {
+                            __threadfence();
+                            k = __ldcg(keys + row);
+                            ft.rowcnt[row] = 0;
+                        }
+                    }
+                    if (complete) {
+                        const int b = static_cast<int>(row / K1);
+                        const int j = static_cast<int>(row - static_cast<long long>(b) * K1);
+                        const int u = used_rows_now(ft, epoch, b);
+                        if (j < u) {
+                            // a row the stream's accept step needs: its word stays for that step, the stream counts it
+                            if (seg == tiles_per_row) keys[row] = k;
+                            __threadfence();               // the word first, then the count
+                            if (atomicAdd(ft.done + b, 1) + 1 == u + ft.prewalk) {
+                                __threadfence();
+                                const int slot = atomicAdd(&sh->q_tail, 1);
+                                if (slot < kQueueCap) st_volatile_s32(queue + slot, b);
+                                else atomicExch(status, kStatusQueueOverflow);   // the host sizes the grid so that this cannot happen
+                            }
+                        } else {
+                            // a row behind the proposal: nothing waits for it, it is reported from here
+                            ft.args.argmax_out[row] = (k != 0ull) ? static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(k)) : 0;
+                            if (seg != tiles_per_row) keys[row] = 0ull;
+                        }
                     }
                 }
             }
@@ -365,7 +457,7 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                 st_volatile_s32(&sh->fin_finished, 1);
             }
             __syncwarp();
-            serve_queue(sam, ft, sh, queue, abort, status, lane);
+            serve_queue(sam, ft, epoch, sh, queue, abort, status, lane);
         }
     } else if (warp > kBulkConsumerWarps + 1) {
         // ------------------------------------------------------------------ walk-ahead warps
@@ -389,14 +481,14 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                     int last = 0;
                     if (lane == 0) {
                         __threadfence();
-                        last = (atomicAdd(ft.done + b, 1) + 1 == ft.expected);
+                        last = (atomicAdd(ft.done + b, 1) + 1 == used_rows_of(ft.args, b) + ft.prewalk);
                     }
                     __syncwarp();
-                    if (__shfl_sync(kFull, last, 0)) fused_accept(sam, ft, b, lane);
+                    if (__shfl_sync(kFull, last, 0)) fused_accept(sam, ft, epoch, b, lane);
                 }
             }
         }
-        if (ft.mode != 0) serve_queue(sam, ft, sh, queue, abort, status, lane);
+        if (ft.mode != 0) serve_queue(sam, ft, epoch, sh, queue, abort, status, lane);
     } else {
         // ------------------------------------------------------------------ consumers
         bool ok = true;
@@ -460,29 +552,26 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             if (warp < kWideGroupWarps) {
                 constexpr int GT = kWideGroupWarps * 32;
                 const int ct = threadIdx.x;
-                long long cur_row = -1;
-                long long row = row_first;
-                int tile = static_cast<int>(t0 - row * tiles_per_row);
                 int s = 0;
                 uint32_t use = 0;
-                for (long long t = t0; t < t1; ++t) {
-                    if (row != cur_row) {
-                        if (cur_row >= 0 && !hand_over(static_cast<int>(cur_row - row_first))) { ok = false; break; }
-                        cur_row = row;
+                for (int i = 0; i < n_rows && ok; ++i) {
+                    const long long row = seq_row(i);
+                    int tile, tile_hi;
+                    tiles_of(row, tile, tile_hi);
+                    for (; tile < tile_hi; ++tile) {
+                        // the outcome of the wait is made uniform so that the warp leaves the loop together
+                        if (!__all_sync(kFull, mbar_wait_bounded(&sh->full[s], use & 1u, abort))) { ok = false; break; }
+                        const int v0 = tile * tile_vec;
+                        const int nv = max(0, min(tile_vec, nvec_row - v0));
+                        const uint4* st = reinterpret_cast<const uint4*>(stage_base + static_cast<size_t>(s) * plan.stage_bytes);
+                        reduce_tile(std::integral_constant<int, GT>{}, st, ct, v0, nv, tile == 0);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sh->empty[s]);
+                        if (ragged != 0 && tile == tiles_per_row - 1) ragged_tail(ct, row);
+                        if (++s == ns) { s = 0; ++use; }
                     }
-                    // the outcome of the wait is made uniform so that the warp leaves the loop together
-                    if (!__all_sync(kFull, mbar_wait_bounded(&sh->full[s], use & 1u, abort))) { ok = false; break; }
-                    const int v0 = tile * tile_vec;
-                    const int nv = max(0, min(tile_vec, nvec_row - v0));
-                    const uint4* st = reinterpret_cast<const uint4*>(stage_base + static_cast<size_t>(s) * plan.stage_bytes);
-                    reduce_tile(std::integral_constant<int, GT>{}, st, ct, v0, nv, tile == 0);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sh->empty[s]);
-                    if (ragged != 0 && tile == tiles_per_row - 1) ragged_tail(ct, row);
-                    if (++tile == tiles_per_row) { tile = 0; ++row; }
-                    if (++s == ns) { s = 0; ++use; }
+                    if (ok && !hand_over(i)) ok = false;
                 }
-                if (ok && cur_row >= 0) ok = hand_over(static_cast<int>(cur_row - row_first));
             }
         } else if (warp < n_cons) {
             // ---- small tiles: groups of four warps take the tiles in turn (tile number `it` of the CTA goes to group
@@ -528,9 +617,17 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             *abort = 1;
             atomicExch(status, kStatusWaitTimeout);
         }
-        if (ft.mode != 0) serve_queue(sam, ft, sh, queue, abort, status, lane);
+        if (ft.mode != 0) serve_queue(sam, ft, epoch, sh, queue, abort, status, lane);
     }
     __syncthreads();
+    if (ft.mode != 0 && threadIdx.x == 0) {
+        // the CTA that leaves last has seen every other CTA read the launch count at its start: it moves the count on
+        __threadfence();
+        if (atomicAdd(ft.launch_words + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+            ft.launch_words[1] = 0;
+            ft.launch_words[0] = epoch;
+        }
+    }
     if (sh->abort) {
         // copies already issued must land before this CTA's shared memory is given up
         if (threadIdx.x == 0) {

@@ -89,7 +89,7 @@ inline int* status_word(unsigned long long* keys, int64_t R) {
 // Partial results land in keys[R]; `status` receives a non-zero code if a kernel gives up on an
 // internal wait.
 // Layout of the verification scratch:
-// keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B] | row_list[R] | list meta words (256 B)
+// keys[R] | status (256 B) | pre_state[B*K] | pre_len[B*K] | done[B] | row_list[R] | list meta words (256 B) | rowcnt[R] | acc_epoch[B]
 struct Scratch {
     unsigned long long* keys;
     int* status;
@@ -98,6 +98,8 @@ struct Scratch {
     int* done;
     int* row_list;
     int* list_meta;
+    int* rowcnt;
+    int* acc_epoch;
     int64_t bytes;
 };
 Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M: automaton slots per stream (walk-ahead arrays)
@@ -113,6 +115,8 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M
     s.done = reinterpret_cast<int*>(p + o);                 o = up(o + static_cast<int64_t>(B) * 4);
     s.row_list = reinterpret_cast<int*>(p + o);             o = up(o + R * 4);
     s.list_meta = reinterpret_cast<int*>(p + o);            o += 256;
+    s.rowcnt = reinterpret_cast<int*>(p + o);               o = up(o + R * 4);
+    s.acc_epoch = reinterpret_cast<int*>(p + o);            o = up(o + static_cast<int64_t>(B) * 4);
     s.bytes = o;
     return s;
 }
@@ -124,7 +128,8 @@ Scratch scratch_layout(void* base, int32_t B, int32_t K, int32_t M = 1) {   // M
 int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsigned long long* keys,
                   int* status, cudaStream_t st, const DeviceSam* sam = nullptr, const PreWalk* pw = nullptr,
                   bool* did_prewalk = nullptr, const AcceptArgs* tail = nullptr, int tail_mode = 0,
-                  int* done = nullptr, bool* did_tail = nullptr, const RowMap* rmap = nullptr) {
+                  int* done = nullptr, bool* did_tail = nullptr, const RowMap* rmap = nullptr, int* rowcnt = nullptr,
+                  int* acc_epoch = nullptr, int* launch_words = nullptr) {
     // Below about 0.8 GB of logits the direct-load kernel followed by an accept kernel that walks the proposal before its
     // grid-dependency wait is the faster pair: it starts sooner than the bulk-copy pipeline and finishes more evenly
     // (measured per step, direct vs bulk-copy: 11.4 vs 13.4 us at B = 4, K = 3; 11.7 vs 13.8 us on the tiny workload;
@@ -161,15 +166,21 @@ int launch_argmax(const void* logits, int64_t stride, int64_t R, int32_t V, unsi
         if (grid < 1) grid = 1;
         const bool prewalk = pw != nullptr && pw->enabled != 0;
         FusedTail ft{};
-        if (tail != nullptr && done != nullptr && g_argmax_variant == 2 && rm.list == nullptr) {
-            // a CTA can be handed at most the streams that overlap its contiguous range of rows
+        if (tail != nullptr && done != nullptr && rowcnt != nullptr && acc_epoch != nullptr && launch_words != nullptr &&
+            g_argmax_variant == 2 &&
+            rm.list == nullptr && plan.n_groups == 1) {
+            // a CTA is handed at most the streams that overlap its contiguous range of rows; it takes the used rows of
+            // that range first, which it can do for up to kOrderCap rows of up to 32 streams
             const int64_t rows_per_cta = (total + grid - 1) / grid / tiles_per_row + 2;
             const int64_t streams_per_cta = rows_per_cta / (tail->K + 1) + 2;
-            const int64_t expected = static_cast<int64_t>(tiles_per_row) * (tail->K + 1) + (prewalk ? 1 : 0);
-            if (streams_per_cta <= kQueueCap && expected < (int64_t(1) << 30)) {
+            if (rows_per_cta <= kOrderCap && streams_per_cta <= 32) {
                 ft.args = *tail;
+                ft.args.flags |= kLeaveUnusedRows;
+                ft.args.acc_epoch = acc_epoch;
+                ft.launch_words = launch_words;
                 ft.done = done;
-                ft.expected = static_cast<int>(expected);
+                ft.rowcnt = rowcnt;
+                ft.prewalk = prewalk ? 1 : 0;
                 ft.mode = tail_mode + 1;
             }
         }
@@ -812,7 +823,7 @@ int sam_verify_ex(const void* logits_bf16, int64_t row_stride_elems, int32_t B, 
     }
     bool did_tail = false;
     rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, nullptr, nullptr, nullptr,
-                       &aa, kTailVerifyOnly, sc.done, &did_tail, &rm);
+                       &aa, kTailVerifyOnly, sc.done, &did_tail, &rm, sc.rowcnt, sc.acc_epoch, sc.list_meta + 8);
     if (rc != SAM_OK) return rc;
     if (!did_tail) {
         rc = launch_accept<kTailVerifyOnly>(DeviceSam{}, aa, st);
@@ -875,7 +886,7 @@ int sam_step_ex(const sam_index* idx,
     }
     bool did_prewalk = false, did_tail = false;
     rc = launch_argmax(logits_bf16, row_stride_elems, R, V, sc.keys, sc.status, st, &idx->dev, &pw, &did_prewalk,
-                       &aa, kTailResume, sc.done, &did_tail, &rm);
+                       &aa, kTailResume, sc.done, &did_tail, &rm, sc.rowcnt, sc.acc_epoch, sc.list_meta + 8);
     if (rc != SAM_OK) return rc;
     if (!did_tail) {
         rc = did_prewalk ? launch_accept<kTailResume>(idx->dev, aa, st) : launch_accept<kTailFullWalk>(idx->dev, aa, st);

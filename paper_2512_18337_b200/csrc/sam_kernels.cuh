@@ -414,6 +414,9 @@ __device__ __forceinline__ long long listed_rows(const RowMap& rm, long long R) 
 
 // Step options (same values as SAM_STEP_* in sam.h).
 constexpr unsigned kNoSpeculation = 1u, kSkipUnusedRows = 2u, kRowListReady = 4u;
+// Internal: the accept step runs inside the argmax kernel as soon as rows 0 .. n_draft are complete; the rows behind the
+// proposal are not its business then (the finisher of the argmax kernel reports them when they are complete).
+constexpr unsigned kLeaveUnusedRows = 0x100u;
 
 // Rows 0..n_draft[b] of every stream, in stream order (n_draft clamped to 0..K, or 0 when speculation
 // is off); one CTA, a block-wide running sum.  meta receives the count and the shape signature.
@@ -584,6 +587,7 @@ struct AcceptArgs {
     unsigned long long* counters;   // [6] running statistics, or nullptr
     int* next_list;           // row list of the NEXT step (rows 0..next_n_draft[b] of every stream, any order), or nullptr
     int* list_meta;           // its meta words (see RowMap)
+    int* acc_epoch;           // [B] number of the launch in which the stream's accept step last ran inside the argmax kernel, or nullptr
 };
 
 // One warp, one stream.  The packed candidates and the walk-ahead results may have been produced
@@ -592,7 +596,7 @@ struct AcceptArgs {
 // does not depend on that kernel's output is loaded first, then the warp waits for it to finish.
 template <int kMode, bool kAfterGrid = false>
 __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const AcceptArgs& p, int b, int lane,
-                                              int* out_a = nullptr, int* out_bonus = nullptr) {
+                                              int* out_a = nullptr, int* out_bonus = nullptr, int epoch = 0) {
     const int K = p.K;
     const int K1 = K + 1;
     const long long row0 = static_cast<long long>(b) * K1;
@@ -632,7 +636,7 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int j = lane + 32 * h;
-        if (j < K1) {
+        if (j < K1 && !((p.flags & kLeaveUnusedRows) && j > nd)) {
             const unsigned long long k = __ldcg(p.keys + row0 + j);
             p.keys[row0 + j] = 0ull;
             // no candidate at all (nothing in the row is greater than -inf): index 0, as a scan from element 0 gives
@@ -696,6 +700,12 @@ __device__ __forceinline__ void accept_stream(const DeviceSam& sam, const Accept
         if (lane == 0) {
             p.state[b] = s;
             p.matched_len[b] = L;
+            if (p.acc_epoch != nullptr) {
+                // inside the argmax kernel: whoever still classifies rows of this stream must not take the next proposal's
+                // length (next_n_draft may be n_draft itself) for this one's
+                p.acc_epoch[b] = epoch;
+                __threadfence();
+            }
             p.next_n_draft[b] = nn;
         }
         if (p.next_list != nullptr) {

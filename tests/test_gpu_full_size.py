@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import oracle
+import paper_2512_18337_b200 as S
 import workload as W
 from harness.cuda_backend import CudaBackend
 from oracle.backend import OracleBackend
@@ -20,7 +21,7 @@ DEV = "cuda:0"
 KEYS = ("argmax", "accepted", "n_accepted", "state", "matched_len", "drafts", "n_draft")
 
 
-def _full_size_closed_loop(i, steps):
+def _full_size_closed_loop(i, steps, variant=0):
     cfg = W.CONFIGS[i].scaled(steps=steps)
     corpus = W.make_corpus(cfg)
     scripts = W.make_scripts(cfg, corpus)
@@ -28,7 +29,11 @@ def _full_size_closed_loop(i, steps):
     assert logits.shape == (cfg.B * (cfg.K + 1), cfg.vocab)
     host_bits = W.device_bits_to_host(logits)
     gpu = CudaBackend(cfg, corpus, logits)
-    tr_g = W.run_closed_loop(cfg, W.ClosedLoopFeeder(cfg, scripts, rowmax), gpu, steps)
+    S.sam_set_argmax_variant(variant)
+    try:
+        tr_g = W.run_closed_loop(cfg, W.ClosedLoopFeeder(cfg, scripts, rowmax), gpu, steps)
+    finally:
+        S.sam_set_argmax_variant(0)
     assert gpu.status() == 0
     del gpu, logits
     torch.cuda.empty_cache()
@@ -46,6 +51,17 @@ def _full_size_closed_loop(i, steps):
 def test_full_size_cfg2_metric_workload():
     """B=256, K=16, min_match=3, 16M-token corpus, 1.32 GB of logits per step."""
     _full_size_closed_loop(2, steps=6)
+
+
+def test_full_size_cfg2_accept_inside_the_argmax_kernel():
+    """The same workload with the accept step of every stream inside the argmax kernel (used rows first, one launch per
+    step), drafts and n_draft rewritten in place while other CTAs still classify rows."""
+    _full_size_closed_loop(2, steps=6, variant=2)
+
+
+def test_full_size_cfg4_accept_inside_the_argmax_kernel():
+    """K = 32: 33 rows per stream, 230 rows per CTA."""
+    _full_size_closed_loop(4, steps=2, variant=2)
 
 
 def test_full_size_cfg3_verify_heavy_with_ties():
