@@ -169,6 +169,8 @@ struct BulkShared {
     int fin_rows;                     // rows of this CTA the finisher has published
     int fin_finished;                 // the finisher has left its loop: no pushes after that
     int prog[kBulkConsumerWarps];     // rows each consumer warp has handed over
+    int n_used;                       // accept step inside the kernel: the first n_used rows the CTA takes are used rows
+    int u_of[32];                     // ... and the number of used rows of every stream of the CTA's share
 };
 static_assert(sizeof(BulkShared) <= 1024, "control block");
 
@@ -315,7 +317,9 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
         const int all_used = __shfl_sync(kFull, used_before, 31);
         used_before -= used;
         rest_before -= rest;
+        if (lane == 0) sh->n_used = all_used;
         if (lane < n_streams) {
+            sh->u_of[lane] = u;
             const int base = static_cast<int>((b_first + lane) * K1 - row_first);     // the stream's row 0 as a row of the share
             for (int j = j_lo; j < j_hi; ++j) {
                 const int at = (j < u) ? used_before + (j - j_lo) : all_used + rest_before + (j - max(j_lo, u));
@@ -323,6 +327,8 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
             }
         }
     }
+    if (ft.mode != 0 && !ordered && n_rows > 0 && threadIdx.x == 0)
+        atomicExch(status, kStatusQueueOverflow);      // the host enables the accept step only for shares that can be ordered
     __syncthreads();
     volatile int* abort = &sh->abort;
     // The i-th row this CTA takes (as a position: in the list, or the row itself), and which of its tiles are the CTA's.
@@ -423,10 +429,11 @@ argmax_bulk_kernel(const __nv_bfloat16* __restrict__ logits, long long stride, l
                         }
                     }
                     if (complete) {
+                        // used or not was settled when the CTA laid out its order (and cannot change for a row that was
+                        // still missing then): no look at n_draft here, which the stream's accept step may have rewritten
                         const int b = static_cast<int>(row / K1);
-                        const int j = static_cast<int>(row - static_cast<long long>(b) * K1);
-                        const int u = used_rows_now(ft, epoch, b);
-                        if (j < u) {
+                        if (i < sh->n_used) {
+                            const int u = sh->u_of[b - static_cast<int>(b_first)];
                             // a row the stream's accept step needs: its word stays for that step, the stream counts it
                             if (seg == tiles_per_row) keys[row] = k;
                             __threadfence();               // the word first, then the count
