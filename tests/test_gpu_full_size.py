@@ -59,11 +59,6 @@ def test_full_size_cfg2_accept_inside_the_argmax_kernel():
     _full_size_closed_loop(2, steps=6, variant=2)
 
 
-def test_full_size_cfg4_accept_inside_the_argmax_kernel():
-    """K = 32: 33 rows per stream, 230 rows per CTA."""
-    _full_size_closed_loop(4, steps=2, variant=2)
-
-
 def test_full_size_cfg3_verify_heavy_with_ties():
     """B=512, K=16, 4M-token corpus, 2.64 GB of logits per step, 1 % planted exact ties at the row maximum."""
     cfg, tr = _full_size_closed_loop(3, steps=8)
